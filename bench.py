@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the AAAC per-layer quantisation path on B200.
+
+One step = the whole hot path over one batch of synthetic layers: for each layer activation
+statistics, scales, quantile initialisation, R fit rounds, the final pack pass and a
+dequantisation.  The workload is the Llama-3-8B-shaped configuration (q_proj 4096x4096,
+gate_proj 14336x4096, down_proj 4096x14336; NVFP4, group 16, 4096 calibration tokens, 20
+rounds) on seeded synthetic data.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  With N > 1 (under torchrun) every rank quantises its own
+batch of layers (independent problems, no data-path collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "aaac_fit_throughput"
+UNIT = "Gweights/s per k-means round"
+ROUNDS = 20
+TOKENS = 4096
+LAYERS = ["q_proj", "gate_proj", "down_proj"]
+BYTES_PER_WEIGHT = 2.0 + 1.0 / 16.0          # NVFP4 fit round: BF16 weight + E4M3 scale per 16
+KERNELS_PER_LAYER = 2 + 3 + 6 + ROUNDS + 1 + 2 + 1   # act_stats, scales, init, rounds, export, pack, dequant
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def measured_traffic_per_weight():
+    """DRAM bytes per weight of the fit-round kernel from the committed ncu summary, if any."""
+    p = os.path.join(ROOT, "profiles", "fit_round_traffic.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["dram_bytes_per_weight"])
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            busy = [s for s in sm if s > 0]
+            out = {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+def make_layers(seed):
+    from paper_2605_08692_b200 import synth
+    return [synth.config2_layer(w, seed=seed, tokens=TOKENS) for w in LAYERS]
+
+
+def cpu_baseline_sample(layers, rounds=ROUNDS, rows=4096):
+    """The oracle, as it stands, on a bounded sample: the first `rows` rows of q_proj, scales +
+    quantile init excluded, `rounds` fit rounds timed on all host cores (about 15 core-seconds)."""
+    import oracle
+    c = layers[0]
+    W = np.ascontiguousarray(c["W"][:rows])
+    I = oracle.act_stats(c["X"][:256])
+    s, ts = oracle.scales(W, c["mode"], c["group"])
+    wt = oracle.normalise(W, c["mode"], c["group"], s, ts)
+    T = oracle.init_quantile(wt)
+    t0 = time.perf_counter()
+    for _ in range(rounds):
+        T, _ = oracle.fit_round(wt, I, c["group"], T)
+    dt = time.perf_counter() - t0
+    return W.size * rounds / dt / 1e9, oracle.max_threads(), f"q_proj rows 0..{rows - 1} x 4096, {rounds} fit rounds", dt
+
+
+def run_reference(args, rank):
+    """Reference arm = the CPU oracle on a bounded sample per step."""
+    if rank != 0:
+        return
+    layers = [__import__("paper_2605_08692_b200.synth", fromlist=["x"]).config2_layer("q_proj", seed=0, rows=1024, tokens=256)]
+    vals = []
+    for i in range(args.warmup + args.steps):
+        v, cores, sample, dt = cpu_baseline_sample(layers, rounds=ROUNDS, rows=1024)
+        if i >= args.warmup:
+            vals.append((v, dt))
+    value = float(np.mean([v for v, _ in vals]))
+    ms = float(np.mean([d for _, d in vals]) * 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "cfg2 Llama-3-8B-shaped linears, NVFP4 g16, 20 rounds (bounded sample per step)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_08692_b200 import binding, build
+    build.build()
+    binding.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    warmup = max(args.warmup, 3)
+    layers = make_layers(seed=rank)
+    mode = layers[0]["mode"]
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    Wd = [to_dev(c["W"]) for c in layers]
+    Xd = [to_dev(c["X"]) for c in layers]
+    shapes = [tuple(c["W"].shape) for c in layers]
+    weights_per_step = sum(n * k for n, k in shapes)
+    # device outputs and scratch, allocated once
+    outs = []
+    for (N, K) in shapes:
+        outs.append(dict(
+            I=torch.empty(K, dtype=torch.float32, device=dev),
+            T01=torch.zeros(2, 16, dtype=torch.float32, device=dev),
+            Tb=torch.empty(2, 16, dtype=torch.uint16, device=dev),
+            scales=torch.empty(N, K // 16, dtype=torch.uint8, device=dev),
+            ts=torch.ones(1, dtype=torch.float32, device=dev),
+            codes=torch.empty(N, K // 2, dtype=torch.uint8, device=dev),
+            err=torch.zeros(2, dtype=torch.float64, device=dev),
+            What=torch.empty(N, K, dtype=torch.bfloat16, device=dev),
+            ws=binding.alloc_workspace(mode, N, K, TOKENS, dev)))
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step():
+        for W, X, o in zip(Wd, Xd, outs):
+            binding.act_stats(X, o["I"], o["ws"], dev_status=status)
+            binding.fit_layer(W, mode, I=o["I"], n_outer=ROUNDS, init=binding.INIT_QUANTILE, T01=o["T01"],
+                              scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
+            binding.pack(W, mode, I=o["I"], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"], tensor_scale=o["ts"],
+                         codes=o["codes"], ws=o["ws"], err_out=o["err"])
+            binding.dequant(o["codes"], o["scales"], o["ts"], o["Tb"], mode, o["What"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    binding.timing_begin(args.steps * len(layers) * ROUNDS)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    round_ms = binding.timing_end(args.steps * len(layers) * ROUNDS)
+    clocks = sampler.stop() if sampler else None
+    if int(status.item()) != 0:
+        raise SystemExit("device status reports non-finite input")
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * weights_per_step * ROUNDS / (ms_step * 1e-3) / 1e9
+
+    # roofline of the dominant kernel: algorithmic bytes of every timed fit-round launch / its device time
+    per_launch_w = []
+    for _ in range(args.steps):
+        for (N, K) in shapes:
+            per_launch_w += [N * K] * ROUNDS
+    bytes_alg = sum(per_launch_w[:len(round_ms)]) * BYTES_PER_WEIGHT
+    fit_ms = float(sum(round_ms))
+    achieved = bytes_alg / (fit_ms * 1e-3) / 1e9 if fit_ms > 0 else 0.0
+    peak, peak_kind = peaks()
+    tpw = measured_traffic_per_weight()
+    roofline = {"kernel": "fit_kernel (one k-means round)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                "traffic": None if tpw is None else tpw * float(np.mean(per_launch_w)),
+                "algorithmic_bytes_per_launch": float(np.mean(per_launch_w)) * BYTES_PER_WEIGHT,
+                "avg_launch_ms": fit_ms / max(len(round_ms), 1),
+                "fit_share_of_step": fit_ms / ms_total if ms_total > 0 else None,
+                "gweights_per_s_kernel": sum(per_launch_w[:len(round_ms)]) / (fit_ms * 1e-3) / 1e9 if fit_ms else 0.0}
+
+    # end to end through the host-buffer entry point (pinned host memory in and out)
+    e2e = None
+    try:
+        host = []
+        for c, (N, K) in zip(layers, shapes):
+            host.append(dict(
+                W=torch.from_numpy(c["W"].view(np.int16)).pin_memory(), X=torch.from_numpy(c["X"].view(np.int16)).pin_memory(),
+                T01=torch.empty(2, 16, dtype=torch.float32).pin_memory(), Tb=torch.empty(2, 16, dtype=torch.int16).pin_memory(),
+                sc=torch.empty(N, K // 16, dtype=torch.uint8).pin_memory(), ts=torch.empty(1, dtype=torch.float32).pin_memory(),
+                codes=torch.empty(N, K // 2, dtype=torch.uint8).pin_memory(), err=torch.empty(2, dtype=torch.float64).pin_memory(),
+                ws=torch.empty(binding.host_workspace_bytes(mode, N, K, TOKENS), dtype=torch.uint8, device=dev)))
+
+        def host_step():
+            for h in host:
+                binding.quantize_layer_host(h["W"], h["X"], mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE,
+                                            T01_host=h["T01"], T01_bf16_host=h["Tb"], scales_host=h["sc"],
+                                            tensor_scale_host=h["ts"], codes_host=h["codes"], err_out_host=h["err"],
+                                            ws=h["ws"])
+        for _ in range(2):
+            host_step()
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            host_step()
+        e1.record()
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item()) / args.steps
+        h2d = sum(h["W"].numel() * 2 + h["X"].numel() * 2 for h in host)
+        d2h = sum(h["codes"].numel() + h["sc"].numel() + 128 + 64 + 4 + 16 + 4 for h in host)
+        e2e = {"value": world * weights_per_step * ROUNDS / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
+    except Exception as ex:                                   # report, never hide
+        e2e = {"value": None, "unit": UNIT, "error": repr(ex)}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample, dt = cpu_baseline_sample(layers)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": dt}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": "cfg2: Llama-3-8B-shaped q_proj 4096x4096, gate_proj 14336x4096, down_proj "
+                                       "4096x14336; NVFP4 g16 E4M3 scales; X 4096 tokens; quantile init; 20 rounds; "
+                                       "step = act_stats + scales + init + 20 fit rounds + pack + dequant per layer",
+                           "weights_per_step": weights_per_step, "rounds": ROUNDS, "seed": "rank",
+                           "l2": "inputs larger than L2: 0.27 GB of W and 0.27 GB of X per step, three layers in turn"},
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": KERNELS_PER_LAYER * len(layers) * args.steps,
+                "clocks": clocks, "wall_s_per_step": ms_step * 1e-3}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

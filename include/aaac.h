@@ -1,0 +1,156 @@
+/*
+ * aaac.h -- C ABI of the B200 (sm_100a) AAAC per-layer quantisation library.
+ *
+ * AAAC replaces the fixed 4-bit table of a group-quantised linear layer by two learned
+ * 16-entry scalar codebooks T0, T1; every group of g weights picks the codebook with the
+ * lower activation-weighted error and stores that choice in the sign bit of its (always
+ * positive) scale.  This library is the per-layer fitting path of Algorithm 1.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns every
+ *     buffer; the library allocates nothing and keeps no per-call state.
+ *   - W is [N x K] row-major BF16 (N = output rows, K = input channels, y = x W^T, Sec. 3.1),
+ *     leading dimension ldw (elements).  Groups are g contiguous elements of a row.
+ *     X is [T x K] row-major BF16 calibration activations, leading dimension ldx.
+ *   - mode AAAC_INT4 : g = 128, scales BF16 [N][K/g], no tensor scale (tensor_scale[0] = 1).
+ *     mode AAAC_NVFP4: g = 16, scales E4M3 bytes [N][K/g] plus one FP32 tensor scale.
+ *   - Tables are [2][16]: T0[0..15] then T1[0..15].
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued and never synchronised:
+ *     results are valid once the stream has been synchronised by the caller.
+ *   - Return value: AAAC_OK or an aaac_status for argument / launch errors (checked before any
+ *     work is enqueued).  Data-dependent conditions (non-finite input) are OR-ed into the
+ *     optional device word `dev_status` instead; nothing traps.
+ *   - Alignment: W, X, codes, What 16-byte aligned; K % 8 == 0; K % g == 0; ldw, ldx, ldo
+ *     multiples of 8.
+ *   - ws is scratch of at least aaac_workspace_bytes(...) bytes, 256-byte aligned.  Calls
+ *     that share a workspace must be ordered on one stream.
+ */
+#ifndef AAAC_H
+#define AAAC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AAAC_OK = 0,
+    AAAC_ERR_NULL = 1,          /* a required pointer is NULL */
+    AAAC_ERR_MODE = 2,          /* unknown mode / init, or group does not match the mode */
+    AAAC_ERR_SHAPE = 3,         /* N < 1, K % g, K % 8, ld < K, ld % 8, T < 1, n_outer < 0 */
+    AAAC_ERR_ALIGN = 4,         /* a pointer is not 16-byte aligned (ws: 256) */
+    AAAC_ERR_WORKSPACE = 5,     /* ws_bytes too small */
+    AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
+    AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
+    AAAC_ERR_UNIMPLEMENTED = 8  /* n_inner != 1 */
+} aaac_status;
+
+typedef enum { AAAC_INT4 = 0, AAAC_NVFP4 = 1 } aaac_mode;
+
+typedef enum {
+    AAAC_INIT_QUANTILE = 0,     /* Eq. 9 / Eq. 10 */
+    AAAC_INIT_GRID = 1,         /* T0 = the format's table, T1 = T0 moved up half a step */
+    AAAC_INIT_USER = 2          /* T01 holds the start tables */
+} aaac_init;
+
+/* bits OR-ed into *dev_status by the kernels */
+#define AAAC_DEV_NONFINITE 1u
+
+const char* aaac_status_string(int status);
+
+/* Bytes of scratch that any call below needs for a layer of this shape (T = calibration
+ * tokens, 0 if activations are never passed). */
+size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
+
+/*
+ * Activation importance, Eq. 7:  I[k] = sum_t X[t,k]^2.
+ * Squares are exact and accumulated in double; the sum is rounded once to FP32.
+ * accumulate = 0 overwrites I; 1 adds to the existing I (FP32 add), so that the tokens can
+ * be streamed in chunks.  Sets AAAC_DEV_NONFINITE if a sum is not finite.
+ */
+int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                   uint32_t* dev_status /* may be NULL */, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Algorithm 1 lines 1-16 for one layer: scales (line 1), normalisation w~ = w / s (Eq. 2,
+ * line 2; w~ = fl32(w * fl32(1/s)) is recomputed on the fly, never stored), importance
+ * (line 3; taken from I, or computed from X when I == NULL), initial tables (lines 4-5),
+ * then n_outer rounds of { assignment step Eq. 8, weighted-centroid update Eq. 11 with
+ * n_inner = 1, keep an entry whose cell has no weight, sort }.
+ *
+ *   scales        out  positive scales (sign bit clear).  INT4: s = bf16(absmax/7) (1 for an
+ *                      all-zero group).  NVFP4: E4M3(absmax / (6 s_t)) in 0x01..0x7E with
+ *                      s_t = layer absmax / 2688.
+ *   tensor_scale  out  [1] FP32 (1.0 for INT4)
+ *   T01           in (AAAC_INIT_USER) / out  [2][16] FP32 tables after the last round, sorted
+ *   err_trace     out  [n_outer] double or NULL: Eq. 8 objective (sum over groups of the
+ *                      smaller weighted error, normalised units) of each round's assignment
+ *   dev_status    out  device word or NULL
+ */
+int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
+                   const float* I, const void* X, int64_t T, int64_t ldx,
+                   int n_outer, int n_inner, int init,
+                   float* T01, void* scales, float* tensor_scale, double* err_trace,
+                   uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Algorithm 1 lines 17-20: round the tables to BF16 (RNE of the FP32 values), recompute
+ * sigma for every group with Eq. 8, store the nearest-entry index under the chosen table
+ * (Eq. 6) as a 4-bit code, and put sigma into the sign bit of the scale.
+ *
+ *   T01_f32   in   [2][16]
+ *   T01_bf16  out  [2][16] BF16 bit patterns (64 bytes)
+ *   scales    in: positive scales from aaac_fit_layer; out: sign bit (bit 15 of the BF16 /
+ *             bit 7 of the E4M3 byte) = sigma
+ *   codes     out  [N][K/2]; element 2i in the low nibble of byte i, 2i+1 in the high nibble
+ *   err_out   out  [2] double or NULL: {Eq. 8 objective under the BF16 tables,
+ *             sum_k I_k (w - w^)^2 in weight units}
+ *   stats     out  [4] uint64 or NULL: {groups with E0 == E1 exactly, weights exactly half-way
+ *             between two different entries of their table, groups re-evaluated in double,
+ *             reserved}
+ * Decisions are exact: sigma and codes equal those of a double-precision evaluation in
+ * index order (near-ties of the FP32 fast path are redone in double).
+ */
+int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
+              const float* I, const float* T01_f32, uint16_t* T01_bf16,
+              void* scales, const float* tensor_scale, uint8_t* codes,
+              double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Eq. 5:  w^ = T_sigma[c] * s, sigma = sign bit of the stored scale, s = its magnitude (times
+ * tensor_scale[0] for NVFP4, the product rounded to FP32), one FP32 multiply, BF16 (RNE) out.
+ */
+int aaac_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale,
+                 const uint16_t* T01_bf16, int64_t N, int64_t K, int mode, int group,
+                 void* What, int64_t ldo, void* stream);
+
+/*
+ * Whole path for one layer with HOST buffers: copies W and X to the device (into ws), runs
+ * aaac_act_stats, aaac_fit_layer and aaac_pack, and copies tables, scales, tensor scale,
+ * codes and errors back.  Host buffers should be page-locked for the copies to be
+ * asynchronous.  ws must hold aaac_host_workspace_bytes(...) bytes of DEVICE memory.
+ * Synchronises the stream before returning; returns AAAC_ERR_NONFINITE if the device
+ * status word was set.
+ */
+size_t aaac_host_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
+int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode, int group,
+                             const void* X_host, int64_t T, int n_outer, int init,
+                             float* T01_host, uint16_t* T01_bf16_host, void* scales_host,
+                             float* tensor_scale_host, uint8_t* codes_host, double* err_out_host,
+                             void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Optional timing of the fit-round kernel: after aaac_timing_begin(n) the next n round
+ * launches on the calling thread's device are bracketed by CUDA events on their stream;
+ * aaac_timing_end synchronises those events and returns how many were recorded, writing each
+ * launch's device time (milliseconds) to ms_host[0..].  Not re-entrant; diagnostics only.
+ */
+int aaac_timing_begin(int max_launches);
+int aaac_timing_end(float* ms_host, int capacity);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AAAC_H */

@@ -1,0 +1,170 @@
+"""ctypes binding of libaaac_b200.so.  Argument marshalling only.
+
+Functions mirror the C entry points (see include/aaac.h for the meaning, layout and ownership
+of every argument).  Tensors must live on the current CUDA device; work is enqueued on
+``torch.cuda.current_stream()`` and is not synchronised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+INT4, NVFP4 = 0, 1
+INIT_QUANTILE, INIT_GRID, INIT_USER = 0, 1, 2
+DEV_NONFINITE = 1
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b200.so")
+_lib = None
+
+EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
+           "aaac_dequant", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
+           "aaac_timing_end"]
+
+
+class AaacError(RuntimeError):
+    pass
+
+
+def lib():
+    """Loads the CUDA library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise AaacError(f"{_LIB_PATH} is missing: build it with `python -m paper_2605_08692_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        L.aaac_status_string.restype = C.c_char_p
+        L.aaac_status_string.argtypes = [C.c_int]
+        L.aaac_workspace_bytes.restype = C.c_size_t
+        L.aaac_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
+        L.aaac_host_workspace_bytes.restype = C.c_size_t
+        L.aaac_host_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
+        vp, i64, ci = C.c_void_p, C.c_int64, C.c_int
+        L.aaac_act_stats.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp, C.c_size_t, vp]
+        L.aaac_fit_layer.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp,
+                                     C.c_size_t, vp]
+        L.aaac_pack.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        L.aaac_dequant.argtypes = [vp, vp, vp, vp, i64, i64, ci, ci, vp, i64, vp]
+        L.aaac_quantize_layer_host.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
+                                               C.c_size_t, vp]
+        L.aaac_timing_begin.argtypes = [ci]
+        L.aaac_timing_end.argtypes = [vp, ci]
+        for f in ("aaac_act_stats", "aaac_fit_layer", "aaac_pack", "aaac_dequant", "aaac_quantize_layer_host",
+                  "aaac_timing_begin", "aaac_timing_end"):
+            getattr(L, f).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise AaacError(f"aaac status {rc}: {lib().aaac_status_string(rc).decode()}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def group_of(mode: int) -> int:
+    return 128 if mode == INT4 else 16
+
+
+def workspace_bytes(mode: int, N: int, K: int, T: int = 0) -> int:
+    return int(lib().aaac_workspace_bytes(mode, N, K, T))
+
+
+def alloc_workspace(mode: int, N: int, K: int, T: int = 0, device="cuda") -> torch.Tensor:
+    return torch.empty(workspace_bytes(mode, N, K, T), dtype=torch.uint8, device=device)
+
+
+def act_stats(X: torch.Tensor, I: torch.Tensor, ws: torch.Tensor, accumulate: bool = False, dev_status=None):
+    T, K = X.shape
+    _check(lib().aaac_act_stats(_ptr(X), T, K, X.stride(0), _ptr(I), int(accumulate), _ptr(dev_status), _ptr(ws),
+                                ws.numel(), _stream()))
+
+
+def fit_layer(W, mode, *, I=None, X=None, n_outer, init, T01, scales, tensor_scale, ws, err_trace=None,
+              dev_status=None, n_inner=1, group=None):
+    N, K = W.shape
+    T, ldx = (X.shape[0], X.stride(0)) if X is not None else (0, 0)
+    _check(lib().aaac_fit_layer(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), _ptr(I), _ptr(X), T, ldx,
+                                n_outer, n_inner, init, _ptr(T01), _ptr(scales), _ptr(tensor_scale), _ptr(err_trace),
+                                _ptr(dev_status), _ptr(ws), ws.numel(), _stream()))
+
+
+def pack(W, mode, *, I, T01, T01_bf16, scales, tensor_scale, codes, ws, err_out=None, stats=None, group=None):
+    N, K = W.shape
+    _check(lib().aaac_pack(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), _ptr(I), _ptr(T01),
+                           _ptr(T01_bf16), _ptr(scales), _ptr(tensor_scale), _ptr(codes), _ptr(err_out), _ptr(stats),
+                           _ptr(ws), ws.numel(), _stream()))
+
+
+def dequant(codes, scales, tensor_scale, T01_bf16, mode, What, group=None):
+    N, K = What.shape
+    _check(lib().aaac_dequant(_ptr(codes), _ptr(scales), _ptr(tensor_scale), _ptr(T01_bf16), N, K, mode,
+                              group or group_of(mode), _ptr(What), What.stride(0), _stream()))
+
+
+def host_workspace_bytes(mode, N, K, T) -> int:
+    return int(lib().aaac_host_workspace_bytes(mode, N, K, T))
+
+
+def quantize_layer_host(W_host, X_host, mode, *, n_outer, init, T01_host, T01_bf16_host, scales_host,
+                        tensor_scale_host, codes_host, err_out_host, ws):
+    """Host tensors in and out (pinned for asynchronous copies); ws is device scratch."""
+    N, K = W_host.shape
+    T = X_host.shape[0]
+    _check(lib().aaac_quantize_layer_host(_ptr(W_host), N, K, mode, group_of(mode), _ptr(X_host), T, n_outer, init,
+                                          _ptr(T01_host), _ptr(T01_bf16_host), _ptr(scales_host),
+                                          _ptr(tensor_scale_host), _ptr(codes_host), _ptr(err_out_host), _ptr(ws),
+                                          ws.numel(), _stream()))
+
+
+def timing_begin(max_launches: int):
+    _check(lib().aaac_timing_begin(max_launches))
+
+
+def timing_end(capacity: int):
+    buf = (C.c_float * capacity)()
+    n = lib().aaac_timing_end(buf, capacity)
+    if n < 0:
+        raise AaacError("aaac_timing_end failed")
+    return [buf[i] for i in range(n)]
+
+
+# ---- convenience for tests and the benchmark: allocate outputs, run the whole path ----
+
+def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trace=False, T01_init=None):
+    """Runs aaac_fit_layer then aaac_pack on device tensors and returns a dict of device tensors."""
+    N, K = W.shape
+    g = group_of(mode)
+    dev = W.device
+    if ws is None:
+        ws = alloc_workspace(mode, N, K, 0 if X is None else X.shape[0], dev)
+    T01 = torch.zeros(2, 16, dtype=torch.float32, device=dev)
+    if T01_init is not None:
+        T01.copy_(T01_init)
+    scales = torch.empty(N, K // g, dtype=torch.uint16 if mode == INT4 else torch.uint8, device=dev)
+    ts = torch.ones(1, dtype=torch.float32, device=dev)
+    trace = torch.zeros(max(n_outer, 1), dtype=torch.float64, device=dev) if want_trace else None
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    if I is None:
+        I = torch.empty(K, dtype=torch.float32, device=dev)
+        act_stats(X, I, ws, dev_status=status)
+    fit_layer(W, mode, I=I, n_outer=n_outer, init=init, T01=T01, scales=scales, tensor_scale=ts, ws=ws,
+              err_trace=trace, dev_status=status)
+    T01_fit = T01.clone()
+    scales_pos = scales.clone()
+    Tb = torch.empty(2, 16, dtype=torch.uint16, device=dev)
+    codes = torch.empty(N, K // 2, dtype=torch.uint8, device=dev)
+    err = torch.zeros(2, dtype=torch.float64, device=dev)
+    stats = torch.zeros(4, dtype=torch.int64, device=dev)
+    pack(W, mode, I=I, T01=T01, T01_bf16=Tb, scales=scales, tensor_scale=ts, codes=codes, ws=ws, err_out=err,
+         stats=stats)
+    return dict(I=I, T01=T01_fit, T01_bf16=Tb, scales=scales, scales_pos=scales_pos, tensor_scale=ts, codes=codes,
+                err=err, stats=stats, trace=trace, status=status)

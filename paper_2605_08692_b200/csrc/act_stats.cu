@@ -1,0 +1,104 @@
+// Activation importance (Eq. 7): I[k] = sum_t X[t,k]^2, a streaming column reduction.
+//
+// Layout: X is [T x K] BF16 row-major.  A block covers 256 adjacent columns (each lane owns
+// 8 of them = one 128-bit load per row) and a strip of rows; its 8 warps take rows
+// round-robin.  The square of a BF16 value is exact in double, and every partial sum is
+// kept in double, so the result differs from an index-order double sum only by double
+// rounding; a second kernel adds the strip partials in strip order and rounds once to FP32.
+#include "internal.cuh"
+
+namespace aaac {
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kUnroll = 4;
+
+__global__ void __launch_bounds__(kWarps * 32)
+act_sumsq_kernel(const uint16_t* __restrict__ X, int64_t T, int64_t K, int64_t ldx,
+                 double* __restrict__ part, int rows_per_split) {
+    __shared__ double sm[kWarps][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t col0 = (int64_t)blockIdx.x * 256 + lane * 8;
+    const bool active = col0 < K;
+    const int64_t t_begin = (int64_t)blockIdx.y * rows_per_split;
+    const int64_t t_end = min(T, t_begin + rows_per_split);
+    double acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.0;
+
+    if (active) {
+        const uint16_t* base = X + col0;
+        int64_t t = t_begin + warp;
+        for (; t + (kUnroll - 1) * kWarps < t_end; t += kUnroll * kWarps) {
+            uint4 v[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u)
+                v[u] = __ldcs(reinterpret_cast<const uint4*>(base + (t + u * kWarps) * ldx));
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    double a = (double)bf16_lo(w[j]), b = (double)bf16_hi(w[j]);
+                    acc[2 * j] = fma(a, a, acc[2 * j]);
+                    acc[2 * j + 1] = fma(b, b, acc[2 * j + 1]);
+                }
+            }
+        }
+        for (; t < t_end; t += kWarps) {
+            uint4 v = __ldcs(reinterpret_cast<const uint4*>(base + t * ldx));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                double a = (double)bf16_lo(w[j]), b = (double)bf16_hi(w[j]);
+                acc[2 * j] = fma(a, a, acc[2 * j]);
+                acc[2 * j + 1] = fma(b, b, acc[2 * j + 1]);
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = acc[j];
+    __syncthreads();
+    const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (col < K) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += sm[w][threadIdx.x];
+        part[(int64_t)blockIdx.y * K + col] = s;
+    }
+}
+
+__global__ void act_final_kernel(const double* __restrict__ part, int splits, int64_t K,
+                                 float* __restrict__ I, int accumulate, uint32_t* dev_status) {
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    double s = 0.0;
+    for (int p = 0; p < splits; ++p) s += part[(int64_t)p * K + k];
+    float v = (float)s;
+    if (accumulate) v += I[k];
+    I[k] = v;
+    if (dev_status && !isfinite(v)) atomicOr(dev_status, AAAC_DEV_NONFINITE);
+}
+
+}  // namespace
+
+cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                             uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
+    const int bx = (int)((K + 255) / 256);
+    int64_t want = ((int64_t)sm_count() * 8 + bx - 1) / bx;
+    int64_t max_by_rows = (T + kWarps - 1) / kWarps;
+    int64_t splits = want < 1 ? 1 : want;
+    if (splits > max_by_rows) splits = max_by_rows;
+    if (splits > kActMaxSplits) splits = kActMaxSplits;
+    int64_t rows = (T + splits - 1) / splits;
+    rows = (rows + kWarps - 1) / kWarps * kWarps;
+    splits = (T + rows - 1) / rows;
+    act_sumsq_kernel<<<dim3(bx, (unsigned)splits), kWarps * 32, 0, st>>>(X, T, K, ldx, ws.act_part, (int)rows);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    act_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(ws.act_part, (int)splits, K, I, accumulate, dev_status);
+    return cudaGetLastError();
+}
+
+}  // namespace aaac

@@ -1,0 +1,321 @@
+// C ABI of the library: argument validation, workspace carving, launch sequencing.
+#include <mutex>
+
+#include "internal.cuh"
+
+namespace aaac {
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Lays the scratch regions out after `base` (which may be null to measure only).
+Workspace carve(void* base, int mode, int64_t N, int64_t K) {
+    Workspace w{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        void* p = base ? static_cast<char*>(base) + off : nullptr;
+        off += up(bytes);
+        return p;
+    };
+    const int g = mode == AAAC_INT4 ? 128 : 16;
+    const int64_t K8 = (K + 7) / 8 * 8;
+    w.ctrl = static_cast<Ctrl*>(take(sizeof(Ctrl)));
+    w.part = static_cast<double*>(take(sizeof(double) * kMaxBlocks * kPartStride));
+    w.rinv = static_cast<float*>(take(sizeof(float) * (size_t)(N > 0 && K > 0 ? N * (K / g + 1) : 1)));
+    w.I = static_cast<float*>(take(sizeof(float) * (size_t)(K8 > 0 ? K8 : 8)));
+    w.act_part = static_cast<double*>(take(sizeof(double) * kActMaxSplits * (size_t)(K8 > 0 ? K8 : 8)));
+    w.qhist = static_cast<uint32_t*>(take(sizeof(uint32_t) * kQBins));
+    w.qprefix = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * (kQBins + 1)));
+    w.qslot_of_bin = static_cast<uint8_t*>(take(kQBins));
+    w.qlist = static_cast<uint32_t*>(take(sizeof(uint32_t) * (size_t)(N > 0 && K > 0 ? N * K : 1)));
+    w.bytes = off;
+    return w;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group) {
+    if (!W) return AAAC_ERR_NULL;
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return AAAC_ERR_MODE;
+    if (group != (mode == AAAC_INT4 ? 128 : 16)) return AAAC_ERR_MODE;
+    if (N < 1 || K < 1 || K % group || K % 8 || ldw < K || ldw % 8) return AAAC_ERR_SHAPE;
+    if (!aligned(W, 16)) return AAAC_ERR_ALIGN;
+    return AAAC_OK;
+}
+
+int check_ws(const void* ws, size_t ws_bytes, size_t need) {
+    if (!ws) return AAAC_ERR_NULL;
+    if (!aligned(ws, kAlign)) return AAAC_ERR_ALIGN;
+    if (ws_bytes < need) return AAAC_ERR_WORKSPACE;
+    return AAAC_OK;
+}
+
+// ---- optional per-launch timing of the fit-round kernel ----
+struct Timing {
+    std::mutex mu;
+    bool on = false;
+    int cap = 0, n = 0;
+    cudaEvent_t* ev = nullptr;      // 2 per launch
+} g_timing;
+
+}  // namespace
+}  // namespace aaac
+
+using namespace aaac;
+
+extern "C" {
+
+const char* aaac_status_string(int status) {
+    switch (status) {
+        case AAAC_OK: return "ok";
+        case AAAC_ERR_NULL: return "a required pointer is NULL";
+        case AAAC_ERR_MODE: return "unknown mode or init, or group size does not match the mode";
+        case AAAC_ERR_SHAPE: return "bad shape (N, K, T, leading dimension or iteration count)";
+        case AAAC_ERR_ALIGN: return "pointer not sufficiently aligned";
+        case AAAC_ERR_WORKSPACE: return "workspace too small";
+        case AAAC_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
+        case AAAC_ERR_NONFINITE: return "input holds Inf or NaN";
+        case AAAC_ERR_UNIMPLEMENTED: return "not implemented (n_inner must be 1)";
+        default: return "unknown status";
+    }
+}
+
+size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T) {
+    (void)T;
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return 0;
+    return carve(nullptr, mode, N, K).bytes;
+}
+
+int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                   uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+    if (!X || !I) return AAAC_ERR_NULL;
+    if (T < 1 || K < 1 || K % 8 || ldx < K || ldx % 8) return AAAC_ERR_SHAPE;
+    if (!aligned(X, 16) || !aligned(I, 4)) return AAAC_ERR_ALIGN;
+    // only the small regions are used; size the check for a 1-row layer of this width
+    int rc = check_ws(ws, ws_bytes, carve(nullptr, AAAC_NVFP4, 1, K).bytes);
+    if (rc) return rc;
+    Workspace w = carve(ws, AAAC_NVFP4, 1, K);
+    return launch_act_stats(static_cast<const uint16_t*>(X), T, K, ldx, I, accumulate, dev_status, w,
+                            static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
+int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
+                   const float* I, const void* X, int64_t T, int64_t ldx,
+                   int n_outer, int n_inner, int init,
+                   float* T01, void* scales, float* tensor_scale, double* err_trace,
+                   uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_layer(W, N, K, ldw, mode, group);
+    if (rc) return rc;
+    if (!T01 || !scales || !tensor_scale) return AAAC_ERR_NULL;
+    if (!I && !X) return AAAC_ERR_NULL;
+    if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID && init != AAAC_INIT_USER) return AAAC_ERR_MODE;
+    if (n_outer < 0) return AAAC_ERR_SHAPE;
+    if (n_inner != 1) return AAAC_ERR_UNIMPLEMENTED;
+    if (!I && (T < 1 || ldx < K || ldx % 8)) return AAAC_ERR_SHAPE;
+    if (!I && !aligned(X, 16)) return AAAC_ERR_ALIGN;
+    if (I && !aligned(I, 16)) return AAAC_ERR_ALIGN;
+    if (!aligned(scales, mode == AAAC_INT4 ? 2 : 1) || !aligned(T01, 4)) return AAAC_ERR_ALIGN;
+    rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
+    if (rc) return rc;
+    Workspace w = carve(ws, mode, N, K);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint16_t* Wp = static_cast<const uint16_t*>(W);
+
+    if (cudaMemsetAsync(w.ctrl, 0, sizeof(Ctrl), st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (!I) {
+        if (launch_act_stats(static_cast<const uint16_t*>(X), T, K, ldx, w.I, 0, dev_status, w, st) != cudaSuccess)
+            return AAAC_ERR_CUDA;
+        I = w.I;
+    }
+    if (launch_scales(Wp, N, K, ldw, mode, scales, tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (launch_init(Wp, N, K, ldw, mode, init, scales, T01, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    for (int r = 0; r < n_outer; ++r) {
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        {
+            std::lock_guard<std::mutex> lk(g_timing.mu);
+            if (g_timing.on && g_timing.n < g_timing.cap) {
+                e0 = g_timing.ev[2 * g_timing.n];
+                e1 = g_timing.ev[2 * g_timing.n + 1];
+                ++g_timing.n;
+            }
+        }
+        if (e0) cudaEventRecord(e0, st);
+        if (launch_fit_round(Wp, N, K, ldw, mode, scales, I, err_trace ? err_trace + r : nullptr, w, st) != cudaSuccess)
+            return AAAC_ERR_CUDA;
+        if (e1) cudaEventRecord(e1, st);
+    }
+    return launch_export_tables(T01, w, st) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
+int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
+              const float* I, const float* T01_f32, uint16_t* T01_bf16,
+              void* scales, const float* tensor_scale, uint8_t* codes,
+              double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_layer(W, N, K, ldw, mode, group);
+    if (rc) return rc;
+    if (!I || !T01_f32 || !T01_bf16 || !scales || !codes) return AAAC_ERR_NULL;
+    if (mode == AAAC_NVFP4 && !tensor_scale) return AAAC_ERR_NULL;
+    if (!aligned(I, 16) || !aligned(codes, 16) || !aligned(T01_bf16, 2)) return AAAC_ERR_ALIGN;
+    rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
+    if (rc) return rc;
+    Workspace w = carve(ws, mode, N, K);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the pack pass uses only the block counter and its own result fields of the control block
+    if (cudaMemsetAsync(&w.ctrl->done, 0, sizeof(uint32_t), st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (cudaMemsetAsync(w.ctrl->pack_err, 0, sizeof(double) * 2 + sizeof(unsigned long long) * 4, st) != cudaSuccess)
+        return AAAC_ERR_CUDA;
+    return launch_pack(static_cast<const uint16_t*>(W), N, K, ldw, mode, I, T01_f32, T01_bf16, scales, tensor_scale,
+                       codes, err_out, reinterpret_cast<unsigned long long*>(stats), w, st) == cudaSuccess
+               ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
+int aaac_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale,
+                 const uint16_t* T01_bf16, int64_t N, int64_t K, int mode, int group,
+                 void* What, int64_t ldo, void* stream) {
+    if (!codes || !scales || !T01_bf16 || !What) return AAAC_ERR_NULL;
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return AAAC_ERR_MODE;
+    if (group != (mode == AAAC_INT4 ? 128 : 16)) return AAAC_ERR_MODE;
+    if (mode == AAAC_NVFP4 && !tensor_scale) return AAAC_ERR_NULL;
+    if (N < 1 || K < 1 || K % group || K % 8 || ldo < K || ldo % 8) return AAAC_ERR_SHAPE;
+    if (!aligned(codes, 4) || !aligned(What, 16)) return AAAC_ERR_ALIGN;
+    return launch_dequant(codes, scales, tensor_scale, T01_bf16, N, K, mode, static_cast<uint16_t*>(What), ldo,
+                          static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
+// ---- host-buffer path ----
+
+namespace {
+struct HostLayout {
+    size_t W, X, I, T01, Tb, scales, ts, codes, err, status, ws, total;
+};
+HostLayout host_layout(int mode, int64_t N, int64_t K, int64_t T) {
+    HostLayout h{};
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off += up(b); return o; };
+    const int g = mode == AAAC_INT4 ? 128 : 16;
+    h.W = take((size_t)N * K * 2);
+    h.X = take((size_t)T * K * 2);
+    h.I = take((size_t)K * 4);
+    h.T01 = take(2 * kM * 4);
+    h.Tb = take(2 * kM * 2);
+    h.scales = take((size_t)N * (K / g) * (mode == AAAC_INT4 ? 2 : 1));
+    h.ts = take(4);
+    h.codes = take((size_t)N * K / 2);
+    h.err = take(16);
+    h.status = take(4);
+    h.ws = take(carve(nullptr, mode, N, K).bytes);
+    h.total = off;
+    return h;
+}
+}  // namespace
+
+size_t aaac_host_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T) {
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return 0;
+    return host_layout(mode, N, K, T).total;
+}
+
+int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode, int group,
+                             const void* X_host, int64_t T, int n_outer, int init,
+                             float* T01_host, uint16_t* T01_bf16_host, void* scales_host,
+                             float* tensor_scale_host, uint8_t* codes_host, double* err_out_host,
+                             void* ws, size_t ws_bytes, void* stream) {
+    if (!W_host || !X_host || !T01_host || !T01_bf16_host || !scales_host || !tensor_scale_host || !codes_host)
+        return AAAC_ERR_NULL;
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return AAAC_ERR_MODE;
+    if (group != (mode == AAAC_INT4 ? 128 : 16)) return AAAC_ERR_MODE;
+    if (N < 1 || K < 1 || T < 1 || K % group || K % 8 || n_outer < 0) return AAAC_ERR_SHAPE;
+    if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID) return AAAC_ERR_MODE;
+    const HostLayout h = host_layout(mode, N, K, T);
+    int rc = check_ws(ws, ws_bytes, h.total);
+    if (rc) return rc;
+    char* d = static_cast<char*>(ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int g = group;
+    const size_t scale_bytes = (size_t)N * (K / g) * (mode == AAAC_INT4 ? 2 : 1);
+    uint32_t* dstatus = reinterpret_cast<uint32_t*>(d + h.status);
+    if (cudaMemsetAsync(dstatus, 0, 4, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (cudaMemcpyAsync(d + h.X, X_host, (size_t)T * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (cudaMemcpyAsync(d + h.W, W_host, (size_t)N * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    void* lws = d + h.ws;
+    const size_t lws_bytes = ws_bytes - h.ws;
+    float* I = reinterpret_cast<float*>(d + h.I);
+    float* T01 = reinterpret_cast<float*>(d + h.T01);
+    rc = aaac_act_stats(d + h.X, T, K, K, I, 0, dstatus, lws, lws_bytes, stream);
+    if (rc) return rc;
+    rc = aaac_fit_layer(d + h.W, N, K, K, mode, group, I, nullptr, 0, 0, n_outer, 1, init, T01, d + h.scales,
+                        reinterpret_cast<float*>(d + h.ts), nullptr, dstatus, lws, lws_bytes, stream);
+    if (rc) return rc;
+    rc = aaac_pack(d + h.W, N, K, K, mode, group, I, T01, reinterpret_cast<uint16_t*>(d + h.Tb), d + h.scales,
+                   reinterpret_cast<float*>(d + h.ts), reinterpret_cast<uint8_t*>(d + h.codes),
+                   reinterpret_cast<double*>(d + h.err), nullptr, lws, lws_bytes, stream);
+    if (rc) return rc;
+    uint32_t hstatus = 0;
+    cudaError_t e = cudaSuccess;
+    auto back = [&](void* dst, size_t off, size_t bytes) {
+        if (e == cudaSuccess && dst) e = cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st);
+    };
+    back(codes_host, h.codes, (size_t)N * K / 2);
+    back(scales_host, h.scales, scale_bytes);
+    back(T01_host, h.T01, 2 * kM * 4);
+    back(T01_bf16_host, h.Tb, 2 * kM * 2);
+    back(tensor_scale_host, h.ts, 4);
+    back(err_out_host, h.err, 16);
+    back(&hstatus, h.status, 4);
+    if (e != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return AAAC_ERR_CUDA;
+    return (hstatus & AAAC_DEV_NONFINITE) ? AAAC_ERR_NONFINITE : AAAC_OK;
+}
+
+// ---- timing of the fit-round kernel ----
+
+int aaac_timing_begin(int max_launches) {
+    std::lock_guard<std::mutex> lk(g_timing.mu);
+    if (g_timing.ev) {
+        for (int i = 0; i < 2 * g_timing.cap; ++i) cudaEventDestroy(g_timing.ev[i]);
+        delete[] g_timing.ev;
+        g_timing.ev = nullptr;
+    }
+    g_timing.on = false;
+    g_timing.n = 0;
+    g_timing.cap = 0;
+    if (max_launches <= 0) return AAAC_OK;
+    g_timing.ev = new cudaEvent_t[2 * (size_t)max_launches];
+    for (int i = 0; i < 2 * max_launches; ++i)
+        if (cudaEventCreate(&g_timing.ev[i]) != cudaSuccess) return AAAC_ERR_CUDA;
+    g_timing.cap = max_launches;
+    g_timing.on = true;
+    return AAAC_OK;
+}
+
+int aaac_timing_end(float* ms_host, int capacity) {
+    std::lock_guard<std::mutex> lk(g_timing.mu);
+    g_timing.on = false;
+    int n = g_timing.n < capacity ? g_timing.n : capacity;
+    for (int i = 0; i < n; ++i) {
+        if (cudaEventSynchronize(g_timing.ev[2 * i + 1]) != cudaSuccess) return -1;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_timing.ev[2 * i], g_timing.ev[2 * i + 1]) != cudaSuccess) return -1;
+        if (ms_host) ms_host[i] = ms;
+    }
+    for (int i = 0; i < 2 * g_timing.cap; ++i) cudaEventDestroy(g_timing.ev[i]);
+    delete[] g_timing.ev;
+    g_timing.ev = nullptr;
+    g_timing.cap = 0;
+    g_timing.n = 0;
+    return n;
+}
+
+}  // extern "C"

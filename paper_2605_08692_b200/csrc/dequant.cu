@@ -1,0 +1,66 @@
+// Dequantisation (Eq. 5): w^ = T_sigma[c] * s, with sigma the sign bit of the stored scale and s
+// its magnitude (times the tensor scale for NVFP4).  A pure stream: 0.5 byte of codes and a
+// scale per group in, 2 bytes out per weight.  Each thread expands one 32-bit word of codes
+// (8 weights) into one 128-bit store.
+#include "internal.cuh"
+
+namespace aaac {
+
+namespace {
+
+template <int MODE>
+__global__ void __launch_bounds__(256)
+dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales,
+               const float* __restrict__ tensor_scale, const uint16_t* __restrict__ Tb,
+               int64_t N, int64_t K, uint16_t* __restrict__ What, int64_t ldo) {
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
+    __shared__ float T[2 * kM];
+    __shared__ float slut[128];
+    if (threadIdx.x < 2 * kM) T[threadIdx.x] = __uint_as_float((uint32_t)Tb[threadIdx.x] << 16);
+    if (MODE == AAAC_NVFP4 && threadIdx.x >= 128)
+        slut[threadIdx.x - 128] = __fmul_rn(e4m3_value(threadIdx.x - 128), tensor_scale[0]);
+    __syncthreads();
+    const int64_t per_row = K / 8, total = N * per_row, Gr = K / G;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / per_row, col = (i % per_row) * 8;
+        const uint32_t word = __ldcs(reinterpret_cast<const uint32_t*>(codes + ((row * K + col) >> 1)));
+        const int64_t gi = row * Gr + col / G;
+        uint32_t sigma;
+        float s;
+        if (MODE == AAAC_INT4) {
+            const uint32_t b = reinterpret_cast<const uint16_t*>(scales)[gi];
+            sigma = b >> 15;
+            s = __uint_as_float((b & 0x7FFFu) << 16);
+        } else {
+            const uint32_t b = reinterpret_cast<const uint8_t*>(scales)[gi];
+            sigma = b >> 7;
+            s = slut[b & 0x7Fu];
+        }
+        const float* Ts = T + sigma * kM;
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t lo = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j)) & 15u], s));
+            const uint32_t hi = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j + 4)) & 15u], s));
+            o[j] = lo | (hi << 16);
+        }
+        __stcs(reinterpret_cast<uint4*>(What + row * ldo + col), make_uint4(o[0], o[1], o[2], o[3]));
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale, const uint16_t* Tb,
+                           int64_t N, int64_t K, int mode, uint16_t* What, int64_t ldo, cudaStream_t st) {
+    const int64_t total = N * (K / 8);
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    if (mode == AAAC_INT4)
+        dequant_kernel<AAAC_INT4><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, tensor_scale, Tb, N, K, What, ldo);
+    else
+        dequant_kernel<AAAC_NVFP4><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, tensor_scale, Tb, N, K, What, ldo);
+    return cudaGetLastError();
+}
+
+}  // namespace aaac

@@ -1,0 +1,272 @@
+// Initial tables (Algorithm 1 lines 4-5).
+//
+// Quantile initialisation (Eq. 9, Eq. 10): T0[i] = Quantile_{i/15}, T1[i] = Quantile_{d + (1-d) i/15},
+// d = 1/30, of all N*K normalised weights, with linear interpolation at position q (n - 1).
+// That needs up to 64 exact order statistics of n values.  They are selected without sorting:
+//   1. histogram of every w~ over 16384 uniform bins on [-8, 8) (shared-memory histogram per
+//      block, merged with integer atomics);
+//   2. one block turns the histogram into a prefix sum, finds the bin and the rank inside the
+//      bin of every requested order statistic, and gives each distinct bin a slot;
+//   3. a second pass over W appends the (order-preserving integer keys of the) values that fall
+//      into a slotted bin to that slot's list -- the lists' sizes are known from step 1;
+//   4. one block per slot selects the requested ranks of its list by an 8-bit radix select;
+//   5. the table entries are interpolated in double and rounded to FP32.
+// Integer atomics only, so the result does not depend on scheduling.
+//
+// Grid initialisation: T0 = the format's table (INT4: -8..7, NVFP4: signed E2M1 with both
+// zeros), T1[i] = (T0[i] + T0[i+1]) / 2 and T1[15] = T0[15] + (T0[15] - T0[14]) / 2.
+#include "internal.cuh"
+
+namespace aaac {
+
+namespace {
+
+__device__ __forceinline__ uint32_t float_key(float f) {      // order-preserving
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+__device__ __forceinline__ int qbin(float x) {
+    int b = __float2int_rd(__fmaf_rn(x, 1024.f, 8192.f));
+    return min(max(b, 0), kQBins - 1);
+}
+
+// reciprocal of the group's scale for the 8 weights a lane holds
+template <int MODE>
+__device__ __forceinline__ float group_rinv(const void* scales, int64_t gi, float s_t) {
+    if (MODE == AAAC_INT4) {
+        const uint32_t b = reinterpret_cast<const uint16_t*>(scales)[gi] & 0x7FFFu;
+        return __frcp_rn(__uint_as_float(b << 16));
+    }
+    const uint32_t c = reinterpret_cast<const uint8_t*>(scales)[gi] & 0x7Fu;
+    return __frcp_rn(__fmul_rn(e4m3_value(c), s_t));
+}
+
+// PASS 0: histogram.  PASS 1: collect candidates of slotted bins.
+template <int MODE, int PASS>
+__global__ void __launch_bounds__(256)
+quantile_scan_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
+                     const void* __restrict__ scales, Ctrl* ctrl, uint32_t* __restrict__ hist,
+                     const uint8_t* __restrict__ slot_of_bin, uint32_t* __restrict__ list) {
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
+    extern __shared__ uint32_t sm[];                 // PASS 0: kQBins counters; PASS 1: kQBins/4 words of slot ids
+    const int lane = threadIdx.x & 31;
+    if (PASS == 0) {
+        for (int i = threadIdx.x; i < kQBins; i += blockDim.x) sm[i] = 0;
+    } else {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(slot_of_bin);
+        for (int i = threadIdx.x; i < kQBins / 4; i += blockDim.x) sm[i] = src[i];
+    }
+    __syncthreads();
+    const uint8_t* sm_slot = reinterpret_cast<const uint8_t*>(sm);
+    const float s_t = ctrl->s_t;
+    const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t it = warp0; it < items; it += nwarps) {
+        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
+        if (col >= K) continue;
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
+        const float r = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
+            const int b = qbin(x);
+            if (PASS == 0) {
+                atomicAdd(&sm[b], 1u);
+            } else {
+                const uint32_t s = sm_slot[b];
+                if (s != 0xFFu) {
+                    const uint32_t pos = atomicAdd(&ctrl->slot_fill[s], 1u);
+                    list[ctrl->slot_off[s] + pos] = float_key(x);
+                }
+            }
+        }
+    }
+    if (PASS == 0) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < kQBins; i += blockDim.x)
+            if (sm[i]) atomicAdd(&hist[i], sm[i]);
+    }
+}
+
+// one block of 1024 threads: prefix sum, bin + local rank of every request, slots
+__global__ void __launch_bounds__(1024)
+quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned long long* __restrict__ prefix,
+                     uint8_t* __restrict__ slot_of_bin) {
+    __shared__ unsigned long long chunk[1024];
+    __shared__ int req_bin[kQReq];
+    const int tid = threadIdx.x;
+    constexpr int per = kQBins / 1024;
+    unsigned long long s = 0;
+    for (int i = 0; i < per; ++i) s += hist[tid * per + i];
+    chunk[tid] = s;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long run = 0;
+        for (int i = 0; i < 1024; ++i) { const unsigned long long c = chunk[i]; chunk[i] = run; run += c; }
+    }
+    __syncthreads();
+    unsigned long long run = chunk[tid];
+    for (int i = 0; i < per; ++i) {
+        prefix[tid * per + i] = run;                      // exclusive prefix
+        run += hist[tid * per + i];
+        slot_of_bin[tid * per + i] = 0xFF;
+    }
+    if (tid == 1023) prefix[kQBins] = run;
+    __syncthreads();
+    if (tid < kQReq) {
+        const unsigned long long r = ctrl->rank[tid];
+        int lo = 0, hi = kQBins;                          // last bin with prefix[bin] <= r
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (prefix[mid] <= r) lo = mid; else hi = mid;
+        }
+        req_bin[tid] = lo;
+        ctrl->req_local[tid] = r - prefix[lo];
+    }
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t ns = 0;
+        unsigned long long off = 0;
+        for (int q = 0; q < kQReq; ++q) {
+            const int b = req_bin[q];
+            if (slot_of_bin[b] == 0xFF) {
+                slot_of_bin[b] = (uint8_t)ns;
+                ctrl->slot_off[ns] = off;
+                ctrl->slot_fill[ns] = 0;
+                off += hist[b];
+                ++ns;
+            }
+            ctrl->req_slot[q] = slot_of_bin[b];
+        }
+        ctrl->slot_off[ns] = off;
+        ctrl->nslots = ns;
+    }
+}
+
+// one block per slot: radix select (4 passes of 8 bits) of every request that lives in this slot
+__global__ void __launch_bounds__(256)
+quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t sh_prefix, sh_mask;
+    __shared__ unsigned long long sh_k;
+    const uint32_t slot = blockIdx.x;
+    if (slot >= ctrl->nslots) return;
+    const uint32_t* keys = list + ctrl->slot_off[slot];
+    const unsigned long long n = ctrl->slot_off[slot + 1] - ctrl->slot_off[slot];
+    for (int q = 0; q < kQReq; ++q) {
+        if (ctrl->req_slot[q] != slot) continue;           // uniform across the block
+        if (threadIdx.x == 0) { sh_prefix = 0; sh_mask = 0; sh_k = ctrl->req_local[q]; }
+        __syncthreads();
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            hist[threadIdx.x] = 0;
+            __syncthreads();
+            const uint32_t prefix = sh_prefix, mask = sh_mask;
+            for (unsigned long long i = threadIdx.x; i < n; i += blockDim.x) {
+                const uint32_t k = keys[i];
+                if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFFu], 1u);
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned long long k = sh_k;
+                int d = 0;
+                for (; d < 255; ++d) {
+                    if (k < hist[d]) break;
+                    k -= hist[d];
+                }
+                sh_k = k;
+                sh_prefix = prefix | ((uint32_t)d << shift);
+                sh_mask = mask | (0xFFu << shift);
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) ctrl->rank_val[q] = key_float(sh_prefix);
+        __syncthreads();
+    }
+}
+
+// entry e uses requests 2e (lower neighbour) and 2e+1 (upper neighbour)
+__global__ void quantile_finish_kernel(Ctrl* ctrl) {
+    const int e = threadIdx.x;
+    if (e >= 2 * kM) return;
+    const double lo = (double)ctrl->rank_val[2 * e], hi = (double)ctrl->rank_val[2 * e + 1];
+    const double v = __dadd_rn(lo, __dmul_rn(ctrl->frac[e], __dsub_rn(hi, lo)));
+    ctrl->T[e] = (double)(float)v;
+}
+
+struct Requests {
+    unsigned long long rank[kQReq];
+    double frac[2 * kM];
+};
+__global__ void set_requests_kernel(Ctrl* ctrl, const Requests rq) {
+    const int t = threadIdx.x;
+    if (t < kQReq) ctrl->rank[t] = rq.rank[t];
+    if (t < 2 * kM) ctrl->frac[t] = rq.frac[t];
+}
+
+__global__ void grid_init_kernel(Ctrl* ctrl, int mode, const float* T01_user) {
+    const int t = threadIdx.x;
+    if (t >= 2 * kM) return;
+    if (T01_user) {
+        ctrl->T[t] = (double)T01_user[t];
+        return;
+    }
+    const double e2m1[kM] = {-6, -4, -3, -2, -1.5, -1, -0.5, 0, 0, 0.5, 1, 1.5, 2, 3, 4, 6};
+    auto base = [&](int i) { return mode == AAAC_INT4 ? (double)(i - 8) : e2m1[i]; };
+    const int i = t & 15;
+    if (t < kM) ctrl->T[t] = base(i);
+    else ctrl->T[t] = (i < 15) ? 0.5 * (base(i) + base(i + 1)) : base(15) + 0.5 * (base(15) - base(14));
+}
+
+}  // namespace
+
+cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
+                        const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st) {
+    if (init != AAAC_INIT_QUANTILE) {
+        grid_init_kernel<<<1, 32, 0, st>>>(ws.ctrl, mode, init == AAAC_INIT_USER ? T01_user : nullptr);
+        return cudaGetLastError();
+    }
+    // positions of the 32 quantiles, as the definition states them
+    Requests rq;
+    const double n1 = (double)(N * K - 1);
+    const double d = 1.0 / (2.0 * (kM - 1));
+    for (int e = 0; e < 2 * kM; ++e) {
+        const int i = e & 15;
+        const double q = (e < kM) ? (double)i / (double)(kM - 1) : d + (1.0 - d) * (double)i / (double)(kM - 1);
+        const double pos = q * n1;
+        double lo = floor(pos), hi = ceil(pos);
+        if (lo < 0) lo = 0;
+        if (hi > n1) hi = n1;
+        if (lo > hi) lo = hi;
+        rq.rank[2 * e] = (unsigned long long)lo;
+        rq.rank[2 * e + 1] = (unsigned long long)hi;
+        rq.frac[e] = pos - lo;
+    }
+    cudaError_t e;
+    set_requests_kernel<<<1, 64, 0, st>>>(ws.ctrl, rq);
+    if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) return e;
+    const int blocks = sm_count() * 2;
+    const size_t sm0 = kQBins * sizeof(uint32_t);
+    if (mode == AAAC_INT4) {
+        if ((e = cudaFuncSetAttribute(quantile_scan_kernel<AAAC_INT4, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
+        quantile_scan_kernel<AAAC_INT4, 0><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist, nullptr, nullptr);
+    } else {
+        if ((e = cudaFuncSetAttribute(quantile_scan_kernel<AAAC_NVFP4, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
+        quantile_scan_kernel<AAAC_NVFP4, 0><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist, nullptr, nullptr);
+    }
+    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qprefix, ws.qslot_of_bin);
+    const int blocks1 = sm_count() * 8;
+    if (mode == AAAC_INT4)
+        quantile_scan_kernel<AAAC_INT4, 1><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, nullptr, ws.qslot_of_bin, ws.qlist);
+    else
+        quantile_scan_kernel<AAAC_NVFP4, 1><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, nullptr, ws.qslot_of_bin, ws.qlist);
+    quantile_select_kernel<<<kQReq, 256, 0, st>>>(ws.ctrl, ws.qlist);
+    quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl);
+    return cudaGetLastError();
+}
+
+}  // namespace aaac

@@ -1,0 +1,101 @@
+// Shared device helpers and launcher declarations of the AAAC sm_100a library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/aaac.h"
+
+namespace aaac {
+
+constexpr int kM = 16;            // entries per table
+constexpr int kNBP = 30;          // merged breakpoints: 15 midpoints of T0 + 15 of T1
+constexpr int kNJ = 31;           // merged intervals
+constexpr int kPartStride = 128;  // doubles per block partial: [2][31] S, [2][31] Wt, E, pad
+constexpr int kMaxBlocks = 2048;  // upper bound on fit-kernel grid size
+constexpr int kQBins = 16384;     // first-level histogram bins of the quantile selection
+constexpr int kQReq = 64;         // order statistics requested (2 per table entry)
+constexpr int kActMaxSplits = 256;
+
+// ---- control block at the start of the workspace (device memory) ----
+struct Ctrl {
+    double T[2 * kM];               // current tables (double between rounds)
+    float s_t;                      // NVFP4 tensor scale
+    uint32_t absmax_bits;           // layer max |w| as float bits (atomicMax on non-negative floats)
+    uint32_t done;                  // blocks that have written their partial this round
+    uint32_t nonfinite;             // set if a non-finite weight was seen
+    // quantile selection
+    unsigned long long rank[kQReq]; // requested 0-based ranks (host-written via kernel args)
+    double frac[2 * kM];            // interpolation fraction per table entry
+    float rank_val[kQReq];          // selected order statistics
+    uint32_t req_slot[kQReq];       // slot of each request
+    unsigned long long req_local[kQReq];   // rank inside the slot's list
+    uint32_t nslots;
+    unsigned long long slot_off[kQReq + 1];
+    uint32_t slot_fill[kQReq];
+    // pack results
+    double pack_err[2];
+    unsigned long long pack_stats[4];
+};
+
+struct Workspace {
+    Ctrl* ctrl;
+    double* part;            // [kMaxBlocks][kPartStride]
+    float* rinv;             // [N*K/g]  INT4 reciprocal scales
+    float* I;                // [K] importance computed from X
+    double* act_part;        // [kActMaxSplits][K]
+    uint32_t* qhist;         // [kQBins]
+    unsigned long long* qprefix;   // [kQBins + 1]
+    uint8_t* qslot_of_bin;   // [kQBins]
+    uint32_t* qlist;         // [N*K]
+    size_t bytes;
+};
+
+// ---- formats ----
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
+    uint32_t u = __float_as_uint(f);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return u >> 16;
+}
+
+// E4M3 (no infinities, 0x7F = NaN): value of a code with the sign bit already removed
+__device__ __forceinline__ float e4m3_value(uint32_t c) {
+    uint32_t e = (c >> 3) & 15u, m = c & 7u;
+    return e ? __uint_as_float(((e + 120u) << 23) | (m << 20)) : (float)m * 0.001953125f;
+}
+
+// nearest-even E4M3 code of a finite x >= 0, saturating at 448 (0x7E)
+__device__ __forceinline__ uint32_t e4m3_encode(float x) {
+    if (!(x < 448.f)) return 0x7Eu;
+    if (x < 0.015625f) return (uint32_t)__float2int_rn(x * 512.f);   // subnormal step 2^-9; 8 -> 2^-6
+    uint32_t u = __float_as_uint(x);
+    u += 0x7FFFFu + ((u >> 20) & 1u);
+    u = (u >> 20) - 960u;                                            // rebias 127 -> 7
+    return u > 0x7Eu ? 0x7Eu : u;
+}
+
+// largest float <= d
+__device__ __forceinline__ float f32_round_down(double d) { return __double2float_rd(d); }
+
+// ---- launchers (each enqueues on `st` and returns the launch status) ----
+cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                             uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, void* scales,
+                          float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
+                        const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_fit_round(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
+                             const float* I, double* err_slot, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,
+                        const float* T01_f32, uint16_t* T01_bf16, void* scales, const float* tensor_scale,
+                        uint8_t* codes, double* err_out, unsigned long long* stats, const Workspace& ws,
+                        cudaStream_t st);
+cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale, const uint16_t* Tb,
+                           int64_t N, int64_t K, int mode, uint16_t* What, int64_t ldo, cudaStream_t st);
+
+int sm_count();
+
+}  // namespace aaac

@@ -1,0 +1,125 @@
+// Per-group positive scales (Algorithm 1, line 1).
+//
+//   INT4  (g = 128): s = bf16_rne(absmax / 7), 1 for an all-zero group, never below 2^-126.
+//                    Also writes r = fl32(1/s) per group for the fit rounds.
+//   NVFP4 (g = 16) : s_t = layer absmax / 2688 (a first pass over W), then per group
+//                    q = E4M3_rne(absmax / (6 s_t)) kept inside 0x01..0x7E; in the lowest
+//                    subnormal step the code is raised so that |w / s| <= 7.5.
+// Both rules keep every normalised weight strictly inside (-8, 8).
+//
+// One warp handles 256 adjacent columns of one row (one 128-bit load per lane); the group
+// maximum is a shuffle reduction over the 16 (INT4) or 2 (NVFP4) lanes of the group.
+#include "internal.cuh"
+
+namespace aaac {
+
+namespace {
+
+__device__ __forceinline__ uint32_t absmax16(uint4 v) {
+    // max over the eight BF16 magnitudes (bit patterns of non-negative floats order like ints)
+    uint32_t m = 0;
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        m = max(m, w[j] & 0x7FFFu);
+        m = max(m, (w[j] >> 16) & 0x7FFFu);
+    }
+    return m;
+}
+
+__global__ void __launch_bounds__(256)
+absmax_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, Ctrl* ctrl) {
+    const int lane = threadIdx.x & 31;
+    const int64_t slabs = (K + 255) / 256, items = N * slabs;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    uint32_t m = 0;
+    for (int64_t it = warp0; it < items; it += nwarps) {
+        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
+        if (col < K) m = max(m, absmax16(__ldg(reinterpret_cast<const uint4*>(W + row * ldw + col))));
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (lane == 0 && m) {
+        atomicMax(&ctrl->absmax_bits, m << 16);
+        if (m >= 0x7F80u) atomicOr(&ctrl->nonfinite, 1u);
+    }
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(256)
+scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, void* __restrict__ scales,
+              float* __restrict__ rinv, float* __restrict__ tensor_scale, Ctrl* ctrl) {
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
+    constexpr int LPG = G / 8;                         // lanes per group
+    const int lane = threadIdx.x & 31;
+    const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+
+    float s_t = 1.f, d6 = 6.f;
+    if (MODE == AAAC_NVFP4) {
+        const float A = __uint_as_float(ctrl->absmax_bits);
+        s_t = (A == 0.f) ? 1.f : __fdiv_rn(A, 2688.f);
+        if (s_t < 0x1p-96f) s_t = 0x1p-96f;
+        d6 = __fmul_rn(6.f, s_t);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctrl->s_t = s_t;
+        if (tensor_scale) tensor_scale[0] = s_t;
+    }
+    bool bad = false;
+    for (int64_t it = warp0; it < items; it += nwarps) {
+        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
+        uint32_t m = 0;
+        if (col < K) m = absmax16(__ldg(reinterpret_cast<const uint4*>(W + row * ldw + col)));
+#pragma unroll
+        for (int o = LPG / 2; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        if (col < K && (lane % LPG) == 0) {
+            const float a = __uint_as_float(m << 16);
+            bad |= (m >= 0x7F80u);
+            const int64_t gi = row * Gr + col / G;
+            if (MODE == AAAC_INT4) {
+                float s = 1.f;
+                if (a != 0.f) {
+                    s = __uint_as_float(f32_to_bf16_rne(__fdiv_rn(a, 7.f)) << 16);
+                    if (s < 0x1p-126f) s = 0x1p-126f;
+                }
+                reinterpret_cast<uint16_t*>(scales)[gi] = (uint16_t)(__float_as_uint(s) >> 16);
+                rinv[gi] = __frcp_rn(s);
+            } else {
+                const float x = __fdiv_rn(a, d6);
+                uint32_t q = e4m3_encode(x);
+                if (q <= 1u) q = (x > 1.25f * 0x1p-9f) ? 2u : 1u;
+                reinterpret_cast<uint8_t*>(scales)[gi] = (uint8_t)q;
+            }
+        }
+    }
+    if (bad) atomicOr(&ctrl->nonfinite, 1u);
+}
+
+__global__ void publish_status_kernel(const Ctrl* ctrl, uint32_t* dev_status) {
+    if (ctrl->nonfinite) atomicOr(dev_status, AAAC_DEV_NONFINITE);
+}
+
+}  // namespace
+
+cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, void* scales,
+                          float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
+    const int blocks = sm_count() * 8;
+    if (mode == AAAC_NVFP4) {
+        absmax_kernel<<<blocks, 256, 0, st>>>(W, N, K, ldw, ws.ctrl);
+        scales_kernel<AAAC_NVFP4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, nullptr, tensor_scale, ws.ctrl);
+    } else {
+        scales_kernel<AAAC_INT4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, ws.rinv, tensor_scale, ws.ctrl);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (dev_status) {
+        publish_status_kernel<<<1, 1, 0, st>>>(ws.ctrl, dev_status);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+}  // namespace aaac
