@@ -44,7 +44,8 @@ typedef enum {
     AAAC_ERR_WORKSPACE = 5,     /* ws_bytes too small */
     AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
     AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
-    AAAC_ERR_UNIMPLEMENTED = 8  /* n_inner != 1 */
+    AAAC_ERR_UNIMPLEMENTED = 8, /* n_inner != 1 */
+    AAAC_ERR_TOO_LARGE = 9      /* size beyond the fixed capacity of a no-allocation entry point */
 } aaac_status;
 
 typedef enum { AAAC_INT4 = 0, AAAC_NVFP4 = 1 } aaac_mode;
@@ -72,6 +73,31 @@ size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
  */
 int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
                    uint32_t* dev_status /* may be NULL */, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * aaac_act_stats for callers that have no scratch buffer to give and must not allocate one.
+ * (The paper has no counterpart: this entry point exists for the integration, not the method.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a serving
+ * engine whose memory pool was sized and handed out at start-up, in a plugin or callback that
+ * is only given its input and output tensors, or on a path that must not stall on cudaMalloc's
+ * implicit synchronisation.  Such a caller cannot create the workspace aaac_act_stats asks for.
+ *
+ * Same inputs, outputs, accumulate flag and result as aaac_act_stats.  The strip partials go
+ * to an 8 MiB array that is part of the library's device image (one copy on every GPU that
+ * loads the library, held until the process exits).  Limits and rules:
+ *   - K <= 32768, otherwise AAAC_ERR_TOO_LARGE is returned and nothing is enqueued;
+ *   - no cudaMalloc / cudaFree or other allocating call is made, on any call;
+ *   - the first call on each device looks up the array's device address (a host-side step
+ *     done once per device, with that device current); make that first call before starting
+ *     any stream capture;
+ *   - all calls on a GPU share the array: calls that may overlap on the GPU (different
+ *     streams without ordering) race on it and give wrong sums.  The array keeps the previous
+ *     call's partials; every value a call reads it has first written itself, so nothing needs
+ *     clearing between calls.
+ */
+int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                           uint32_t* dev_status /* may be NULL */, void* stream);
 
 /*
  * Algorithm 1 lines 1-16 for one layer: scales (line 1), normalisation w~ = w / s (Eq. 2,

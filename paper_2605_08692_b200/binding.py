@@ -19,7 +19,7 @@ _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b2
 _lib = None
 
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
-           "aaac_dequant", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
+           "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end"]
 
 
@@ -42,6 +42,8 @@ def lib():
         L.aaac_host_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
         vp, i64, ci = C.c_void_p, C.c_int64, C.c_int
         L.aaac_act_stats.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp, C.c_size_t, vp]
+        L.aaac_act_stats_noalloc.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp]
+        L.aaac_act_stats_noalloc.restype = ci
         L.aaac_fit_layer.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp,
                                      C.c_size_t, vp]
         L.aaac_pack.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
@@ -86,6 +88,14 @@ def act_stats(X: torch.Tensor, I: torch.Tensor, ws: torch.Tensor, accumulate: bo
     T, K = X.shape
     _check(lib().aaac_act_stats(_ptr(X), T, K, X.stride(0), _ptr(I), int(accumulate), _ptr(dev_status), _ptr(ws),
                                 ws.numel(), _stream()))
+
+
+def act_stats_noalloc(X: torch.Tensor, I: torch.Tensor, accumulate: bool = False, dev_status=None):
+    """aaac_act_stats without a workspace: for callers that may not allocate device memory.
+    K <= 32768; calls on one GPU share the library's built-in scratch and must not overlap."""
+    T, K = X.shape
+    _check(lib().aaac_act_stats_noalloc(_ptr(X), T, K, X.stride(0), _ptr(I), int(accumulate), _ptr(dev_status),
+                                        _stream()))
 
 
 def fit_layer(W, mode, *, I=None, X=None, n_outer, init, T01, scales, tensor_scale, ws, err_trace=None,

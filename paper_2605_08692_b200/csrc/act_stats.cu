@@ -5,6 +5,8 @@
 // round-robin.  The square of a BF16 value is exact in double, and every partial sum is
 // kept in double, so the result differs from an index-order double sum only by double
 // rounding; a second kernel adds the strip partials in strip order and rounds once to FP32.
+#include <mutex>
+
 #include "internal.cuh"
 
 namespace aaac {
@@ -102,3 +104,70 @@ cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ld
 }
 
 }  // namespace aaac
+
+// ---------------------------------------------------------------------------------------------
+// aaac_act_stats_noalloc: the same reduction for callers that cannot hand over scratch memory.
+//
+// The strip partials live in a fixed array in the library's own device image instead of a
+// caller workspace, so the call needs no buffer besides X and I.  The array exists once per
+// GPU that loads the library and is shared by every call on that GPU.
+// ---------------------------------------------------------------------------------------------
+namespace aaac {
+namespace {
+
+constexpr int kNoAllocMaxK = 32768;       // widest layer input the built-in scratch covers
+constexpr int kNoAllocSplits = 32;        // row strips (8 MiB of scratch in total)
+
+static __device__ __align__(256) double g_noalloc_part[(size_t)kNoAllocSplits * kNoAllocMaxK];
+
+std::mutex g_noalloc_mu;
+double* g_noalloc_ptr[64] = {nullptr};   // device address of the array, per device ordinal
+
+// Host code cannot use the array's name as a pointer: the name only identifies the symbol.
+// Its device address is looked up once per device, with that device current.
+cudaError_t noalloc_scratch(double** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        double* p = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_part);
+        if (e != cudaSuccess) return e;
+        if (!p) return cudaErrorInvalidSymbol;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace aaac
+
+extern "C" int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
+                                      uint32_t* dev_status, void* stream) {
+    using namespace aaac;
+    if (!X || !I) return AAAC_ERR_NULL;
+    if (T < 1 || K < 1 || K % 8 || ldx < K || ldx % 8) return AAAC_ERR_SHAPE;
+    if (K > kNoAllocMaxK) return AAAC_ERR_TOO_LARGE;
+    if ((reinterpret_cast<uintptr_t>(X) % 16) || (reinterpret_cast<uintptr_t>(I) % 4)) return AAAC_ERR_ALIGN;
+    double* part = nullptr;
+    if (noalloc_scratch(&part) != cudaSuccess) return AAAC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int bx = (int)((K + 255) / 256);
+    int64_t splits = ((int64_t)sm_count() * 8 + bx - 1) / bx;
+    const int64_t max_by_rows = (T + kWarps - 1) / kWarps;
+    if (splits > max_by_rows) splits = max_by_rows;
+    if (splits > kNoAllocSplits) splits = kNoAllocSplits;
+    if (splits < 1) splits = 1;
+    int64_t rows = (T + splits - 1) / splits;
+    rows = (rows + kWarps - 1) / kWarps * kWarps;
+    splits = (T + rows - 1) / rows;
+    // every partial that the second kernel reads is written by the first: nothing has to be cleared
+    act_sumsq_kernel<<<dim3(bx, (unsigned)splits), kWarps * 32, 0, st>>>(static_cast<const uint16_t*>(X), T, K, ldx,
+                                                                        part, (int)rows);
+    if (cudaGetLastError() != cudaSuccess) return AAAC_ERR_CUDA;
+    act_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(part, (int)splits, K, I, accumulate, dev_status);
+    return cudaGetLastError() == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}

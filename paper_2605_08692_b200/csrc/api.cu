@@ -90,6 +90,7 @@ const char* aaac_status_string(int status) {
         case AAAC_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
         case AAAC_ERR_NONFINITE: return "input holds Inf or NaN";
         case AAAC_ERR_UNIMPLEMENTED: return "not implemented (n_inner must be 1)";
+        case AAAC_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this no-allocation entry point";
         default: return "unknown status";
     }
 }
