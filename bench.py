@@ -104,9 +104,9 @@ class ClockSampler:
         return out
 
 
-def make_layers(seed):
+def make_layers(seed, names=None):
     from paper_2605_08692_b200 import synth
-    return [synth.config2_layer(w, seed=seed, tokens=TOKENS) for w in LAYERS]
+    return [synth.config2_layer(w, seed=seed, tokens=TOKENS) for w in (names or LAYERS)]
 
 
 def cpu_baseline_sample(layers, rounds=ROUNDS, rows=4096):
@@ -154,6 +154,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", default=",".join(LAYERS),
+                    help="subset of the workload's layers (profiling a small case); the default is the full workload")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -177,7 +179,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     warmup = max(args.warmup, 3)
-    layers = make_layers(seed=rank)
+    names = [n for n in args.layers.split(",") if n]
+    layers = make_layers(seed=rank, names=names)
     mode = layers[0]["mode"]
 
     def to_dev(a):
@@ -304,9 +307,10 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
                 "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic",
-                "config": {"workload": "cfg2: Llama-3-8B-shaped q_proj 4096x4096, gate_proj 14336x4096, down_proj "
-                                       "4096x14336; NVFP4 g16 E4M3 scales; X 4096 tokens; quantile init; 20 rounds; "
-                                       "step = act_stats + scales + init + 20 fit rounds + pack + dequant per layer",
+                "config": {"workload": ("cfg2: Llama-3-8B-shaped q_proj 4096x4096, gate_proj 14336x4096, down_proj "
+                                        "4096x14336; NVFP4 g16 E4M3 scales; X 4096 tokens; quantile init; 20 rounds; "
+                                        "step = act_stats + scales + init + 20 fit rounds + pack + dequant per layer")
+                           if names == LAYERS else "cfg2 SUBSET (not the benchmark workload): " + ",".join(names),
                            "weights_per_step": weights_per_step, "rounds": ROUNDS, "seed": "rank",
                            "l2": "inputs larger than L2: 0.27 GB of W and 0.27 GB of X per step, three layers in turn"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
