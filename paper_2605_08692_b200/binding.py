@@ -15,7 +15,7 @@ INT4, NVFP4 = 0, 1
 INIT_QUANTILE, INIT_GRID, INIT_USER = 0, 1, 2
 DEV_NONFINITE = 1
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b200.so")
+_LIB_PATH = os.environ.get("AAAC_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b200.so")
 _lib = None
 
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",

@@ -7,8 +7,8 @@ import sys
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
-LIB = os.path.join(_DIR, "libaaac_b200.so")
-SOURCES = ["api.cu", "act_stats.cu", "scales.cu", "init.cu", "fit.cu", "dequant.cu"]
+LIB = os.environ.get("AAAC_B200_LIB") or os.path.join(_DIR, "libaaac_b200.so")
+SOURCES = ["api.cu", "act_stats.cu", "scales.cu", "init.cu", "fit.cu", "pack.cu", "dequant.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "--fmad=true", "-prec-div=true", "-prec-sqrt=true", "-ftz=false"]
 
@@ -24,7 +24,7 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+        cmd = [nvcc] + NVCC_FLAGS + os.environ.get("AAAC_NVCC_EXTRA", "").split() + (["-Xptxas", "-v"] if verbose else []) + \
               [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
         subprocess.check_call(cmd)
     return LIB

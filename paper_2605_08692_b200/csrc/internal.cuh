@@ -16,6 +16,14 @@ constexpr int kQBins = 16384;     // first-level histogram bins of the quantile 
 constexpr int kQReq = 64;         // order statistics requested (2 per table entry)
 constexpr int kActMaxSplits = 256;
 
+// shape of the fit-round kernel: warps per block, copies of the {J_low, thr} table
+#ifndef AAAC_FIT_WARPS
+#define AAAC_FIT_WARPS 4
+#endif
+#ifndef AAAC_FIT_REP
+#define AAAC_FIT_REP 16
+#endif
+
 // ---- control block at the start of the workspace (device memory) ----
 struct Ctrl {
     double T[2 * kM];               // current tables (double between rounds)
