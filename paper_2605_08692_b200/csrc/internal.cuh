@@ -10,7 +10,7 @@ namespace aaac {
 constexpr int kM = 16;            // entries per table
 constexpr int kNBP = 30;          // merged breakpoints: 15 midpoints of T0 + 15 of T1
 constexpr int kNJ = 31;           // merged intervals
-constexpr int kPartStride = 128;  // doubles per block partial: [2][31] S, [2][31] Wt, E, pad
+constexpr int kPartStride = 128;  // doubles per block partial (pack: [2][31] S, Wt, E; fit: [32] S, [32] Wt, E)
 constexpr int kMaxBlocks = 2048;  // upper bound on fit-kernel grid size
 constexpr int kQBins = 16384;     // first-level histogram bins of the quantile selection
 constexpr int kQReq = 64;         // order statistics requested (2 per table entry)
@@ -18,10 +18,10 @@ constexpr int kActMaxSplits = 256;
 
 // shape of the fit-round kernel: warps per block, copies of the {J_low, thr} table
 #ifndef AAAC_FIT_WARPS
-#define AAAC_FIT_WARPS 4
+#define AAAC_FIT_WARPS 12
 #endif
 #ifndef AAAC_FIT_REP
-#define AAAC_FIT_REP 16
+#define AAAC_FIT_REP 8
 #endif
 
 // ---- control block at the start of the workspace (device memory) ----
