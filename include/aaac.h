@@ -58,6 +58,7 @@ typedef enum {
 
 /* bits OR-ed into *dev_status by the kernels */
 #define AAAC_DEV_NONFINITE 1u
+#define AAAC_DEV_TIMEOUT 2u      /* a bounded wait inside a kernel ran out; results are not valid */
 
 const char* aaac_status_string(int status);
 
@@ -168,8 +169,9 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
                              void* ws, size_t ws_bytes, void* stream);
 
 /*
- * Optional timing of the fit-round kernel: after aaac_timing_begin(n) the next n round
- * launches on the calling thread's device are bracketed by CUDA events on their stream;
+ * Optional timing of the fit-rounds kernel: after aaac_timing_begin(n) the next n launches of
+ * it (one per aaac_fit_layer call with n_outer > 0, covering all rounds of that call) on the
+ * calling thread's device are bracketed by CUDA events on their stream;
  * aaac_timing_end synchronises those events and returns how many were recorded, writing each
  * launch's device time (milliseconds) to ms_host[0..].  Not re-entrant; diagnostics only.
  */

@@ -34,7 +34,7 @@ Workspace carve(void* base, int mode, int64_t N, int64_t K) {
     const int g = mode == AAAC_INT4 ? 128 : 16;
     const int64_t K8 = (K + 7) / 8 * 8;
     w.ctrl = static_cast<Ctrl*>(take(sizeof(Ctrl)));
-    w.part = static_cast<double*>(take(sizeof(double) * kMaxBlocks * kPartStride));
+    w.part = static_cast<double*>(take(sizeof(double) * 2 * kMaxBlocks * kPartStride));
     w.rinv = static_cast<float*>(take(sizeof(float) * (size_t)(N > 0 && K > 0 ? N * (K / g + 1) : 1)));
     w.I = static_cast<float*>(take(sizeof(float) * (size_t)(K8 > 0 ? K8 : 8)));
     w.act_part = static_cast<double*>(take(sizeof(double) * kActMaxSplits * (size_t)(K8 > 0 ? K8 : 8)));
@@ -144,9 +144,10 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
     }
     if (launch_scales(Wp, N, K, ldw, mode, scales, tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
     if (launch_init(Wp, N, K, ldw, mode, init, scales, T01, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
-    for (int r = 0; r < n_outer; ++r) {
+    {
+        // all rounds run in one launch; the optional timing brackets that launch
         cudaEvent_t e0 = nullptr, e1 = nullptr;
-        {
+        if (n_outer > 0) {
             std::lock_guard<std::mutex> lk(g_timing.mu);
             if (g_timing.on && g_timing.n < g_timing.cap) {
                 e0 = g_timing.ev[2 * g_timing.n];
@@ -155,7 +156,7 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
             }
         }
         if (e0) cudaEventRecord(e0, st);
-        if (launch_fit_round(Wp, N, K, ldw, mode, scales, I, err_trace ? err_trace + r : nullptr, w, st) != cudaSuccess)
+        if (launch_fit_rounds(Wp, N, K, ldw, mode, scales, I, n_outer, err_trace, dev_status, w, st) != cudaSuccess)
             return AAAC_ERR_CUDA;
         if (e1) cudaEventRecord(e1, st);
     }

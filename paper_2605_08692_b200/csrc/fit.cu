@@ -1,13 +1,21 @@
-// One fit round (Algorithm 1 lines 6-16 with n_inner = 1): assignment step (Eq. 8) and
-// activation-weighted centroid update (Eq. 11) in a single pass over W.
+// The fit rounds (Algorithm 1 lines 6-16 with n_inner = 1): per round the assignment step
+// (Eq. 8) and the activation-weighted centroid update (Eq. 11) in a single pass over W.  All
+// rounds of a layer run in ONE persistent kernel (one block per SM, cooperative launch): after
+// its pass every block publishes a partial, the blocks meet at a grid-wide barrier, and every
+// block adds all partials in the same fixed order, so each holds the same new tables without a
+// second barrier or a relaunch.  The barrier wait is bounded: if it runs out, the kernel sets
+// AAAC_DEV_TIMEOUT in the device status word and returns.
 //
 // Per weight the kernel needs (a) the interval J of the merged breakpoint list of both tables
 // that holds w~ = fl32(w * r) (Eq. 2) -- J fixes the nearest entry of T0 and of T1 (Eq. 4) --
 // (b) its two weighted squared errors, and (c) one accumulation into the centroid sums of cell
 // (sigma, J).
 //
-// (a) Interval.  Uniform bins of width 1/64 on (-8, 8): bin = low 10 bits of
-//     fl32(64 x + 1.5 * 2^23 + 512).  A table gives per bin {J_low, thr}: J_low breakpoints lie
+// (a) Interval.  Uniform bins of width 1/64 on (-8, 8): the mantissa of
+//     fl32(64 x + 512 + 1.5 * 2^(23-k)) holds (64 x + 512) * 2^k rounded to an integer; masked,
+//     it is the byte offset bin * 2^k of the bin's table entry (2^k = bytes per bin over all
+//     copies), bin = floor of 64 x + 512 after rounding to a multiple of 2^-k.
+//     A table gives per bin {J_low, thr}: J_low breakpoints lie
 //     below the bin, thr is the one breakpoint inside it (+inf if none), J = J_low + (x > thr).
 //     Breakpoints are the rounded-down FP32 midpoints, for which x > thr <=> x > midpoint, so J
 //     is exact.  A bin that holds two or more breakpoints points at a poisoned slot (J = 31)
@@ -27,9 +35,10 @@
 //     (sum I (x - c), sum I) with c the constant of (b) for the entry the weight is assigned to,
 //     so the new entry is c + sum I (x - c) / sum I.  The residual sums are small and of mixed
 //     sign, which keeps the FP32 accumulation error some 20 times below that of sum I x.  No
-//     atomics, fixed order.  One partial per block; the last block to finish adds the partials
-//     in a fixed order, forms the centroids, keeps entries of empty cells, sorts, and stores the
-//     new tables and the Eq. 8 objective of the round (sum over groups of the smaller error).
+//     atomics, fixed order.  One partial per block and round; after the barrier the partials are
+//     added in a fixed order, the centroids formed (entries of empty cells keep their value) and
+//     sorted; block 0 stores the Eq. 8 objective of the round (sum over groups of the smaller
+//     error) and, after the last round, the tables.
 //
 // Tables in shared memory are replicated to cut bank conflicts: the {J_low, thr} table REP
 // times (lane l uses copy l mod REP), the {P, Q} table and the bins once per lane (conflict
@@ -51,22 +60,21 @@ constexpr int kNBins = 1024;
 constexpr int kJSlots = 32;                        // 31 intervals + the poisoned slot
 constexpr int kSlotBytes = 32 * 8;                 // one 8-byte entry per lane
 constexpr int kPoison = kNJ * kSlotBytes;          // byte offset of the poisoned slot
-constexpr float kMagic = 12582912.f + 512.f;       // 1.5 * 2^23 + 512
 constexpr int kCells = 2 * kM;                     // bins per lane: [sigma][entry]
 constexpr int kUsed = 2 * kCells + 1;              // [32] S, [32] Wt, E
 constexpr uint32_t kIdxMask = 15u;                 // low mantissa bits of a centre constant = entry index
 
-// Shared-memory accesses of the hot loop with explicit 32-bit addresses.  The table loads are
-// plain asm (the tables are not written while the main loop runs, so they may move freely);
-// the bin accesses are volatile, which keeps every read-modify-write in program order.
+// Shared-memory accesses of the hot loop with explicit 32-bit addresses.  All are volatile asm,
+// which keeps them in the order in which the loop writes them (table lookups of one row issued
+// ahead of the read-modify-write chain of the previous one).
 __device__ __forceinline__ uint2 lds_table_u2(uint32_t addr) {
     uint2 r;
-    asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(addr));
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(addr));
     return r;
 }
 __device__ __forceinline__ float2 lds_table_f2(uint32_t addr) {
     float2 r;
-    asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
     return r;
 }
 __device__ __forceinline__ float2 lds_bin(uint32_t addr) {
@@ -85,7 +93,6 @@ struct FitTables {
     float tmp_b[32];
     uint8_t tmp_src[32];
     uint8_t src[32];
-    uint8_t idx0[32], idx1[32];   // canonical (lowest duplicate) entry index on interval J
     float rlut[128];              // NVFP4: fl32(1 / s_eff) per E4M3 code
     float2 pq32[kJSlots];         // {P, Q} of every interval before replication
     float centre[2 * kM];         // centre constant of every entry (index in the low 4 mantissa bits)
@@ -101,18 +108,18 @@ struct FitParams {
     const float* rinv;            // INT4 reciprocal scales
     const float* I;
     Ctrl* ctrl;
-    double* part;
-    double* err_slot;
+    double* part;                 // [2][kMaxBlocks][kPartStride]: partials of even / odd rounds
+    double* err_trace;            // [n_rounds] or null
+    uint32_t* dev_status;         // or null
+    int n_rounds;
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
 };
 
-// Builds every lookup table of the round from the current tables in the control block.
+// Builds every lookup table of the round from the current tables in S.Td.
 template <int MODE, int NW, int REP>
-__device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dyn) {
+__device__ void build_tables(FitTables& S, unsigned char* dyn) {
     constexpr int NT = NW * 32;
     const int tid = threadIdx.x;
-    if (tid < 2 * kM) S.Td[tid] = p.ctrl->T[tid];
-    __syncthreads();
     if (tid < kNBP) {
         const int r = tid / 15, i = tid % 15;
         const double mid = (S.Td[r * kM + i] + S.Td[r * kM + i + 1]) * 0.5;
@@ -120,9 +127,13 @@ __device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dy
         S.tmp_src[tid] = (uint8_t)r;
     }
     if (tid >= 30 && tid < 32) S.bp[tid] = __int_as_float(0x7F800000);
-    if (MODE == AAAC_NVFP4 && tid < 128) {
-        const float s = __fmul_rn(e4m3_value((uint32_t)tid), p.ctrl->s_t);
-        S.rlut[tid] = tid ? __frcp_rn(s) : 0.f;
+    if (tid >= 32 && tid < 32 + 2 * kM) {
+        // centre constant: FP32 rounding of the entry with its canonical (lowest duplicate) index
+        // in the low mantissa bits
+        const int t = tid - 32, r = t & 16;
+        int i = t & 15;
+        while (i > 0 && S.Td[r + i - 1] == S.Td[r + i]) --i;
+        S.centre[t] = __uint_as_float((__float_as_uint((float)S.Td[t]) & ~kIdxMask) | (uint32_t)i);
     }
     __syncthreads();
     if (tid < kNBP) {
@@ -133,14 +144,6 @@ __device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dy
         S.src[rank] = S.tmp_src[tid];
     }
     __syncthreads();
-    if (tid < 2 * kM) {
-        // canonical (lowest duplicate) index of the entry, carried in the low mantissa bits
-        int i = tid & 15;
-        const int r = tid & 16;
-        while (i > 0 && S.Td[r + i - 1] == S.Td[r + i]) --i;
-        S.centre[tid] = __uint_as_float((__float_as_uint((float)S.Td[tid]) & ~kIdxMask) | (uint32_t)i);
-    }
-    __syncthreads();
     float2* lut2 = reinterpret_cast<float2*>(dyn + (size_t)REP * kNBins * 8);
     if (tid < kJSlots) {
         float P = __int_as_float(0x7FC00000), Q = P;
@@ -149,15 +152,11 @@ __device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dy
             for (int j = 0; j < tid; ++j) { i0 += (S.src[j] == 0); i1 += (S.src[j] == 1); }
             while (i0 > 0 && S.Td[i0 - 1] == S.Td[i0]) --i0;
             while (i1 > 0 && S.Td[kM + i1 - 1] == S.Td[kM + i1]) --i1;
-            S.idx0[tid] = (uint8_t)i0;
-            S.idx1[tid] = (uint8_t)i1;
             S.PQ[tid] = make_double2(S.Td[i0], S.Td[kM + i1]);
             P = S.centre[i0];
             Q = S.centre[kM + i1];
         } else {
             S.PQ[tid] = make_double2(0.0, 0.0);
-            S.idx0[tid] = 0;
-            S.idx1[tid] = 0;
         }
         double tm = fabs(S.Td[tid]);                     // 32 entries, one per lane of warp 0
 #pragma unroll
@@ -165,26 +164,22 @@ __device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dy
         if (tid == 0) S.tmax283 = __double2float_ru(tm * (2.83 * 32.0));
         S.pq32[tid] = make_float2(P, Q);
     }
-    __syncthreads();
-    for (int i = tid; i < kJSlots * 32; i += NT) lut2[i] = S.pq32[i >> 5];
-    // {J_low, thr} per bin; bin b holds the x with 64 x + 512 in [b - 1/2, b + 1/2]
+    // {J_low, thr} per bin.  Bin b holds the x with 64 x + 512 in [b - h, b + 1 - h], h = half of
+    // the rounding step 1 / (8 REP) of the bin arithmetic.  The breakpoints are sorted, so those
+    // inside a bin are the first ones not below its lower edge.
     uint2* lut1 = reinterpret_cast<uint2*>(dyn);
+    constexpr float h = 0.5f / (float)(REP * 8);
     for (int b = tid; b < kNBins; b += NT) {
-        const float lo = ((float)b - 512.5f) * 0.015625f, hi = ((float)b - 511.5f) * 0.015625f;
-        int below = 0, inside = 0;
-        float thr = __int_as_float(0x7F800000);
-        for (int j = 0; j < kNBP; ++j) {
-            const float v = S.bp[j];
-            below += (v < lo);
-            if (v >= lo && v <= hi) {
-                if (inside == 0) thr = v;
-                ++inside;
-            }
-        }
+        const float lo = ((float)b - 512.f - h) * 0.015625f, hi = ((float)b - 511.f - h) * 0.015625f;
+        int below = 0;                                   // number of breakpoints < lo (binary search)
+#pragma unroll
+        for (int step = 16; step; step >>= 1)
+            if (below + step <= kNBP && S.bp[below + step - 1] < lo) below += step;
+        const float v0 = S.bp[below], v1 = S.bp[below + 1];     // bp[30], bp[31] = +inf
         uint2 e;
-        if (inside <= 1) {
+        if (!(v1 <= hi)) {                               // at most one breakpoint inside
             e.x = (uint32_t)(below * kSlotBytes);
-            e.y = __float_as_uint(thr);
+            e.y = v0 <= hi ? __float_as_uint(v0) : 0x7F800000u;
         } else {
             e.x = (uint32_t)kPoison;
             e.y = 0x7F800000u;
@@ -192,6 +187,8 @@ __device__ void build_tables(FitTables& S, const FitParams& p, unsigned char* dy
 #pragma unroll
         for (int c = 0; c < REP; ++c) lut1[b * REP + c] = e;
     }
+    __syncthreads();
+    for (int i = tid; i < kJSlots * 32; i += NT) lut2[i] = S.pq32[i >> 5];
     __syncthreads();
 }
 
@@ -229,8 +226,37 @@ __device__ __noinline__ Exact8 exact_groups(const FitTables* S, Row8 r, int need
     return out;
 }
 
+constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
+
+// Grid-wide barrier of a cooperative launch: block arrivals are counted in ctrl->bar, which only
+// grows during a launch.  Returns false (in every thread of the block) if the wait ran out or
+// another block has given up; the caller then leaves the kernel.
+__device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        atomicAdd(&ctrl->bar, 1u);
+        bool good = true;
+        for (unsigned spins = 0;; ++spins) {
+            unsigned seen, abort;
+            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->bar) : "memory");
+            if (seen >= target) break;
+            asm volatile("ld.relaxed.gpu.u32 %0, [%1];" : "=r"(abort) : "l"(&ctrl->abort) : "memory");
+            if (abort || spins >= kBarrierSpinLimit) {
+                atomicExch(&ctrl->abort, 1u);
+                good = false;
+                break;
+            }
+            __nanosleep(64);
+        }
+        S.is_last = good;
+    }
+    __syncthreads();
+    return S.is_last != 0;
+}
+
 template <int MODE, int NW, int REP>
-__global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p) {
+__global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;
     constexpr int R = kRowsPerWarp;
@@ -244,8 +270,6 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
     __shared__ FitTables S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    build_tables<MODE, NW, REP>(S, p, dyn);
-
     // 32-bit shared addresses.  Slot offsets carry the address of this lane's column of the
     // {P, Q} table, so a lookup there needs no further arithmetic.
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
@@ -253,9 +277,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
     const int c0 = (int)(sm_base + kLut1Bytes + lane * 8), c1 = c0 + kSlotBytes;       // + J * 256
     const uint32_t bins_warp = sm_base + kLut1Bytes + kLut2Bytes + warp * kBinBytes;
     const uint32_t bins_lane = bins_warp + lane * 8;                                   // + cell * 256
-    for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
-    const float tmax283 = S.tmax283;
-    double Eacc = 0.0;
+    double* wsum = reinterpret_cast<double*>(dyn);         // [NW][kPartStride], over the first table
 
     // 32-bit index arithmetic throughout (N, K < 2^31); only the final element offsets are 64-bit
     const int N = (int)p.N, K = (int)p.K;
@@ -283,6 +305,24 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
             }
         }
     };
+
+    if (tid < 2 * kM) S.Td[tid] = p.ctrl->T[tid];
+    if (MODE == AAAC_NVFP4 && tid >= 64 && tid < 192) {
+        const int c = tid - 64;
+        const float sv = __fmul_rn(e4m3_value((uint32_t)c), p.ctrl->s_t);
+        S.rlut[c] = c ? __frcp_rn(sv) : 0.f;
+    }
+    __syncthreads();
+
+    // bin arithmetic: the masked mantissa of fl32(64 x + kMagic) is bin * (REP * 8)
+    constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
+    constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
+
+  for (int round = 0; round < p.n_rounds; ++round) {
+    build_tables<MODE, NW, REP>(S, dyn);
+    for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
+    const float tmax283 = S.tmax283;
+    double Eacc = 0.0;
 
     int cur_slab = -1;
     float Iv[8];
@@ -326,27 +366,39 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
             isum *= 1.0001f;
         }
         const int row0 = rb * kRowsPerItem + warp * R;
+        const int nrows = min(R, N - row0);                // rows of this warp inside the layer (may be <= 0)
 
-#pragma unroll
-        for (int u = 0; u < R; ++u) {
-            if (row0 + u >= N) break;                      // rows past N (uniform over the warp)
-            // ---- lookups and both weighted errors of the row
+        // The rows of the item go through three stages, written out in the order in which the
+        // shared-memory operations are to be issued, so that the read-modify-write chain on the
+        // bins of one row runs while the table lookups of the next row are in flight:
+        //   L1(u): w~ and the loads of {J_low, thr};   L2(u): slot and the loads of {P, Q};
+        //   M(u):  errors, sigma, the centred terms and bin addresses;   B(u): bins += terms.
+        float x[8];                                        // w~ of the row in L1..M
+        uint2 e1v[8];                                      // {J_low * 256, thr}
+        float2 pq[8];                                      // {P, Q}
+        float mt[8];                                       // chosen centred term I (x - c) of the row in B
+        uint32_t ba[8];                                    // its bin address
+        auto L1 = [&](int u) {
             const float rinv = MODE == AAAC_NVFP4 ? S.rlut[sc[u] & 0x7Fu] : __uint_as_float(sc[u]);
             const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
+                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) & kBinMask;
+                e1v[j] = lds_table_u2(lut1_lane + off);
+            }
+        };
+        auto L2 = [&]() {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                pq[j] = lds_table_f2(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
+        };
+        auto M = [&](int u) {
             float m0[8], m1[8];
-            uint32_t cb0[8], cb1[8];                       // bits of the two centre constants
             float e0 = 0.f, e1 = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
-                const float x = __fmul_rn(wf, rinv);
-                const uint32_t bin = (uint32_t)__float_as_int(__fmaf_rn(x, 64.f, kMagic)) & (kNBins - 1);
-                const uint2 e = lds_table_u2(lut1_lane + bin * (REP * 8));
-                const uint32_t o = e.x + (uint32_t)((x > __uint_as_float(e.y)) ? c1 : c0);
-                const float2 pq = lds_table_f2(o);
-                cb0[j] = __float_as_uint(pq.x);
-                cb1[j] = __float_as_uint(pq.y);
-                const float u0 = __fsub_rn(x, pq.x), u1 = __fsub_rn(x, pq.y);
+                const float u0 = __fsub_rn(x[j], pq[j].x), u1 = __fsub_rn(x[j], pq[j].y);
                 m0[j] = __fmul_rn(Iv[j], u0);
                 m1[j] = __fmul_rn(Iv[j], u1);
                 e0 = __fmaf_rn(m0[j], u0, e0);
@@ -359,7 +411,9 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
             }
             const float es = e0 + e1;
             const float tau = 0x1p-24f * __fmaf_rn(tmax283, __fsqrt_ru(__fmul_ru(isum, es)), 16.f * es);
-            const bool near = col_ok && !(fabsf(e1 - e0) > tau);
+            // lanes past K carry I = 0 and w~ = 0; they need the exact path only if their slot is
+            // poisoned (NaN), so that no NaN reaches a bin
+            const bool near = !(fabsf(e1 - e0) > tau) && (col_ok || !(es == es));
             bool sg = e1 < e0;
             double emin = (double)(sg ? e1 : e0);
             if (__any_sync(0xFFFFFFFFu, near)) {
@@ -367,34 +421,80 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
                 // this lane's centred terms from the intervals that call has found
                 Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    r.x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                    r.I[j] = Iv[j];
-                }
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = Iv[j]; }
                 const Exact8 ex = exact_groups<LPG>(&S, r, (int)near);
                 if (near) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const float2 pq = lds_table_f2((uint32_t)(c0 + ex.J[j] * kSlotBytes));
-                        cb0[j] = __float_as_uint(pq.x);
-                        cb1[j] = __float_as_uint(pq.y);
-                        m0[j] = __fmul_rn(Iv[j], __fsub_rn(r.x[j], pq.x));
-                        m1[j] = __fmul_rn(Iv[j], __fsub_rn(r.x[j], pq.y));
+                        pq[j] = lds_table_f2((uint32_t)(c0 + ex.J[j] * kSlotBytes));
+                        m0[j] = __fmul_rn(Iv[j], __fsub_rn(x[j], pq[j].x));
+                        m1[j] = __fmul_rn(Iv[j], __fsub_rn(x[j], pq[j].y));
                     }
                     sg = ex.sigma != 0;
                     emin = ex.emin;
                 }
             }
             if (col_ok && (lane % LPG) == 0) Eacc += emin;
-            // ---- centroid sums of the row: cell = entry index under the chosen table
+            // cell = entry index (low bits of the centre constant) under the chosen table
             const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint32_t addr = base + ((sg ? cb1[j] : cb0[j]) & kIdxMask) * kSlotBytes;
-                float2 a = lds_bin(addr);
-                a.x += sg ? m1[j] : m0[j];
+                mt[j] = sg ? m1[j] : m0[j];
+                ba[j] = base + (__float_as_uint(sg ? pq[j].y : pq[j].x) & kIdxMask) * kSlotBytes;
+            }
+        };
+        auto B = [&](int j0, int j1) {
+#pragma unroll
+            for (int j = j0; j < j1; ++j) {
+                float2 a = lds_bin(ba[j]);
+                a.x += mt[j];
                 a.y += Iv[j];
-                sts_bin(addr, a);
+                sts_bin(ba[j], a);
+            }
+        };
+
+        if (nrows == R) {
+            // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
+            L1(0);
+            L2();
+            M(0);
+#pragma unroll
+            for (int u = 1; u < R; ++u) {
+                float mt_prev[8];
+                uint32_t ba_prev[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { mt_prev[j] = mt[j]; ba_prev[j] = ba[j]; }
+                auto Bprev = [&](int j0, int j1) {
+#pragma unroll
+                    for (int j = j0; j < j1; ++j) {
+                        float2 a = lds_bin(ba_prev[j]);
+                        a.x += mt_prev[j];
+                        a.y += Iv[j];
+                        sts_bin(ba_prev[j], a);
+                    }
+                };
+                L1(u);
+                Bprev(0, 4);
+                L2();
+                Bprev(4, 8);
+                M(u);
+            }
+            B(0, 8);
+        } else {
+            // ragged last row block of the layer: row by row
+            for (int u = 0; u < nrows; ++u) {
+                // (u is uniform over the warp; the stages index v[] and sc[] with it)
+                uint4 vv = v[0];
+                uint32_t ss = sc[0];
+#pragma unroll
+                for (int t = 1; t < R; ++t)
+                    if (u == t) { vv = v[t]; ss = sc[t]; }
+                v[0] = vv;
+                sc[0] = ss;
+                L1(0);
+                L2();
+                M(0);
+                B(0, 8);
             }
         }
     }
@@ -402,7 +502,6 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
     // ---- block partial: lane c of a warp adds the 32 lane-private values of cell c (in a
     //      rotated, fixed order that avoids bank conflicts); then the warps are added ----
     __syncthreads();                                       // every warp is done with the lookup tables
-    double* wsum = reinterpret_cast<double*>(dyn);         // [NW][kPartStride], over the first table
     {
         double sx = 0.0, sy = 0.0;
 #pragma unroll 4
@@ -418,30 +517,29 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
     for (int s = 16; s; s >>= 1) Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, s);
     if (lane == 0) wsum[warp * kPartStride + 2 * kCells] = Eacc;
     __syncthreads();
+    double* part = p.part + (size_t)(round & 1) * kMaxBlocks * kPartStride;
     if (tid < kUsed) {
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < NW; ++w) s += wsum[w * kPartStride + tid];
-        p.part[(int64_t)blockIdx.x * kPartStride + tid] = s;
+        part[(size_t)blockIdx.x * kPartStride + tid] = s;
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) S.is_last = (atomicAdd(&p.ctrl->done, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!S.is_last) return;
 
-    // ---- last block: add the partials of all blocks in a fixed order (NT / 128 interleaved
-    //      strands per value, each in block order, then the strands in order), update the tables ----
-    __threadfence();
+    // ---- all blocks meet; then each adds the partials of all blocks in the same fixed order
+    //      (kStrands interleaved strands per value, each in block order, then the strands) ----
+    if (!grid_barrier(S, p.ctrl, (unsigned)(round + 1) * gridDim.x)) {
+        if (blockIdx.x == 0 && tid == 0 && p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
+        return;
+    }
     {
-        constexpr int kStrands = NT / 128;
-        const int val = tid & 127, strand = tid >> 7;
-        double s = 0.0;
-        if (val < kUsed) {
+        constexpr int kStrands = NT / kUsed;
+        const int strand = tid / kUsed, val = tid - strand * kUsed;
+        if (strand < kStrands) {
+            double s = 0.0;
 #pragma unroll 8
-            for (unsigned b = strand; b < gridDim.x; b += kStrands) s += __ldcg(p.part + (int64_t)b * kPartStride + val);
+            for (unsigned b = strand; b < gridDim.x; b += kStrands) s += __ldcg(part + (size_t)b * kPartStride + val);
+            wsum[strand * kPartStride + val] = s;
         }
-        wsum[strand * kPartStride + val] = s;
         __syncthreads();
         if (tid < kUsed) {
             double t = 0.0;
@@ -451,24 +549,26 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_round_kernel(const FitParams p
         }
     }
     __syncthreads();
+    double tnew = 0.0;
+    int rank = 0;
     if (tid < 2 * kM) {
         // cells of duplicate entries are empty: they keep their value
         const double sx = S.tot[tid], wt = S.tot[kCells + tid];
-        const double t = (wt > 0.0) ? (double)S.centre[tid] + __ddiv_rn(sx, wt) : S.Td[tid];
+        tnew = (wt > 0.0) ? (double)S.centre[tid] + __ddiv_rn(sx, wt) : S.Td[tid];
         // ascending order within the table by rank (ties by index)
         const int r = tid & 16;
-        int rank = 0;
         for (int i = 0; i < kM; ++i) {
             const double sxi = S.tot[r + i], wti = S.tot[kCells + r + i];
             const double ti = (wti > 0.0) ? (double)S.centre[r + i] + __ddiv_rn(sxi, wti) : S.Td[r + i];
-            rank += (ti < t) || (ti == t && i < (tid & 15));
+            rank += (ti < tnew) || (ti == tnew && i < (tid & 15));
         }
-        p.ctrl->T[r + rank] = t;
     }
-    if (tid == 0) {
-        if (p.err_slot) *p.err_slot = S.tot[2 * kCells];
-        p.ctrl->done = 0;
-    }
+    __syncthreads();
+    if (tid < 2 * kM) S.Td[(tid & 16) + rank] = tnew;
+    if (blockIdx.x == 0 && tid == 0 && p.err_trace) p.err_trace[round] = S.tot[2 * kCells];
+    __syncthreads();
+  }
+    if (blockIdx.x == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
 }
 
 __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
@@ -476,23 +576,26 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
 }
 
 template <int MODE, int NW, int REP>
-cudaError_t launch_variant(const FitParams& p, unsigned grid, cudaStream_t st) {
+cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)REP * kNBins * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
-    auto kern = fit_round_kernel<MODE, NW, REP>;
+    auto kern = fit_rounds_kernel<MODE, NW, REP>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, NW * 32, smem, st>>>(p);
-    return cudaGetLastError();
+    void* args[] = {&p};
+    // cooperative: every block is resident, which the grid-wide barrier relies on
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(NW * 32), args, smem, st);
 }
 
 }  // namespace
 
-cudaError_t launch_fit_round(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
-                             const float* I, double* err_slot, const Workspace& ws, cudaStream_t st) {
+cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
+                              const float* I, int n_rounds, double* err_trace, uint32_t* dev_status,
+                              const Workspace& ws, cudaStream_t st) {
+    if (n_rounds <= 0) return cudaSuccess;
     FitParams p{};
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
     p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
-    p.ctrl = ws.ctrl; p.part = ws.part; p.err_slot = err_slot;
+    p.ctrl = ws.ctrl; p.part = ws.part; p.err_trace = err_trace; p.dev_status = dev_status; p.n_rounds = n_rounds;
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
     const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;

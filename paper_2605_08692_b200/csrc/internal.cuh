@@ -31,6 +31,8 @@ struct Ctrl {
     uint32_t absmax_bits;           // layer max |w| as float bits (atomicMax on non-negative floats)
     uint32_t done;                  // blocks that have written their partial this round
     uint32_t nonfinite;             // set if a non-finite weight was seen
+    uint32_t bar;                   // block arrivals at the grid barrier of the fit-rounds kernel
+    uint32_t abort;                 // set when a barrier wait ran out
     // quantile selection
     unsigned long long rank[kQReq]; // requested 0-based ranks (host-written via kernel args)
     double frac[2 * kM];            // interpolation fraction per table entry
@@ -47,7 +49,7 @@ struct Ctrl {
 
 struct Workspace {
     Ctrl* ctrl;
-    double* part;            // [kMaxBlocks][kPartStride]
+    double* part;            // [2][kMaxBlocks][kPartStride]
     float* rinv;             // [N*K/g]  INT4 reciprocal scales
     float* I;                // [K] importance computed from X
     double* act_part;        // [kActMaxSplits][K]
@@ -94,8 +96,9 @@ cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, 
                           float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
                         const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st);
-cudaError_t launch_fit_round(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
-                             const float* I, double* err_slot, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
+                              const float* I, int n_rounds, double* err_trace, uint32_t* dev_status,
+                              const Workspace& ws, cudaStream_t st);
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,
                         const float* T01_f32, uint16_t* T01_bf16, void* scales, const float* tensor_scale,
