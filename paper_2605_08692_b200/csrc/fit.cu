@@ -49,57 +49,11 @@
 // bitwise reproducible.  A warp takes 4 rows; each lane 8 adjacent columns (one 128-bit load
 // per row), so its eight importances stay in registers.  A group is 2 lanes (g = 16) or 16
 // lanes (g = 128).  The next item's rows are loaded while the current item is processed.
-#include "internal.cuh"
+#include "lookup.cuh"
 
 namespace aaac {
 
 namespace {
-
-constexpr int kRowsPerWarp = 4;
-constexpr int kNBins = 1024;
-constexpr int kJSlots = 32;                        // 31 intervals + the poisoned slot
-constexpr int kSlotBytes = 32 * 8;                 // one 8-byte entry per lane
-constexpr int kPoison = kNJ * kSlotBytes;          // byte offset of the poisoned slot
-constexpr int kCells = 2 * kM;                     // bins per lane: [sigma][entry]
-constexpr int kUsed = 2 * kCells + 1;              // [32] S, [32] Wt, E
-constexpr uint32_t kIdxMask = 15u;                 // low mantissa bits of a centre constant = entry index
-
-// Shared-memory accesses of the hot loop with explicit 32-bit addresses.  All are volatile asm,
-// which keeps them in the order in which the loop writes them (table lookups of one row issued
-// ahead of the read-modify-write chain of the previous one).
-__device__ __forceinline__ uint2 lds_table_u2(uint32_t addr) {
-    uint2 r;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(addr));
-    return r;
-}
-__device__ __forceinline__ float2 lds_table_f2(uint32_t addr) {
-    float2 r;
-    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
-    return r;
-}
-__device__ __forceinline__ float2 lds_bin(uint32_t addr) {
-    float2 r;
-    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr) : "memory");
-    return r;
-}
-__device__ __forceinline__ void sts_bin(uint32_t addr, float2 v) {
-    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" :: "r"(addr), "f"(v.x), "f"(v.y) : "memory");
-}
-
-struct FitTables {
-    double Td[2 * kM];
-    double2 PQ[kJSlots];          // nearest entries of T0 / T1 on interval J, as double
-    float bp[32];                 // sorted breakpoints, bp[30] = bp[31] = +inf
-    float tmp_b[32];
-    uint8_t tmp_src[32];
-    uint8_t src[32];
-    float rlut[128];              // NVFP4: fl32(1 / s_eff) per E4M3 code
-    float2 pq32[kJSlots];         // {P, Q} of every interval before replication
-    float centre[2 * kM];         // centre constant of every entry (index in the low 4 mantissa bits)
-    float tmax283;                // 2.83 * 32 * max |entry|, rounded up
-    int is_last;
-    double tot[kPartStride];
-};
 
 struct FitParams {
     const uint16_t* W;
@@ -114,117 +68,6 @@ struct FitParams {
     int n_rounds;
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
 };
-
-// Builds every lookup table of the round from the current tables in S.Td.
-template <int MODE, int NW, int REP>
-__device__ void build_tables(FitTables& S, unsigned char* dyn) {
-    constexpr int NT = NW * 32;
-    const int tid = threadIdx.x;
-    if (tid < kNBP) {
-        const int r = tid / 15, i = tid % 15;
-        const double mid = (S.Td[r * kM + i] + S.Td[r * kM + i + 1]) * 0.5;
-        S.tmp_b[tid] = f32_round_down(mid);
-        S.tmp_src[tid] = (uint8_t)r;
-    }
-    if (tid >= 30 && tid < 32) S.bp[tid] = __int_as_float(0x7F800000);
-    if (tid >= 32 && tid < 32 + 2 * kM) {
-        // centre constant: FP32 rounding of the entry with its canonical (lowest duplicate) index
-        // in the low mantissa bits
-        const int t = tid - 32, r = t & 16;
-        int i = t & 15;
-        while (i > 0 && S.Td[r + i - 1] == S.Td[r + i]) --i;
-        S.centre[t] = __uint_as_float((__float_as_uint((float)S.Td[t]) & ~kIdxMask) | (uint32_t)i);
-    }
-    __syncthreads();
-    if (tid < kNBP) {
-        const float b = S.tmp_b[tid];
-        int rank = 0;
-        for (int j = 0; j < kNBP; ++j) rank += (S.tmp_b[j] < b) || (S.tmp_b[j] == b && j < tid);
-        S.bp[rank] = b;
-        S.src[rank] = S.tmp_src[tid];
-    }
-    __syncthreads();
-    float2* lut2 = reinterpret_cast<float2*>(dyn + (size_t)REP * kNBins * 8);
-    if (tid < kJSlots) {
-        float P = __int_as_float(0x7FC00000), Q = P;
-        if (tid < kNJ) {
-            int i0 = 0, i1 = 0;
-            for (int j = 0; j < tid; ++j) { i0 += (S.src[j] == 0); i1 += (S.src[j] == 1); }
-            while (i0 > 0 && S.Td[i0 - 1] == S.Td[i0]) --i0;
-            while (i1 > 0 && S.Td[kM + i1 - 1] == S.Td[kM + i1]) --i1;
-            S.PQ[tid] = make_double2(S.Td[i0], S.Td[kM + i1]);
-            P = S.centre[i0];
-            Q = S.centre[kM + i1];
-        } else {
-            S.PQ[tid] = make_double2(0.0, 0.0);
-        }
-        double tm = fabs(S.Td[tid]);                     // 32 entries, one per lane of warp 0
-#pragma unroll
-        for (int o = 16; o; o >>= 1) tm = fmax(tm, __shfl_xor_sync(0xFFFFFFFFu, tm, o));
-        if (tid == 0) S.tmax283 = __double2float_ru(tm * (2.83 * 32.0));
-        S.pq32[tid] = make_float2(P, Q);
-    }
-    // {J_low, thr} per bin.  Bin b holds the x with 64 x + 512 in [b - h, b + 1 - h], h = half of
-    // the rounding step 1 / (8 REP) of the bin arithmetic.  The breakpoints are sorted, so those
-    // inside a bin are the first ones not below its lower edge.
-    uint2* lut1 = reinterpret_cast<uint2*>(dyn);
-    constexpr float h = 0.5f / (float)(REP * 8);
-    for (int b = tid; b < kNBins; b += NT) {
-        const float lo = ((float)b - 512.f - h) * 0.015625f, hi = ((float)b - 511.f - h) * 0.015625f;
-        int below = 0;                                   // number of breakpoints < lo (binary search)
-#pragma unroll
-        for (int step = 16; step; step >>= 1)
-            if (below + step <= kNBP && S.bp[below + step - 1] < lo) below += step;
-        const float v0 = S.bp[below], v1 = S.bp[below + 1];     // bp[30], bp[31] = +inf
-        uint2 e;
-        if (!(v1 <= hi)) {                               // at most one breakpoint inside
-            e.x = (uint32_t)(below * kSlotBytes);
-            e.y = v0 <= hi ? __float_as_uint(v0) : 0x7F800000u;
-        } else {
-            e.x = (uint32_t)kPoison;
-            e.y = 0x7F800000u;
-        }
-#pragma unroll
-        for (int c = 0; c < REP; ++c) lut1[b * REP + c] = e;
-    }
-    __syncthreads();
-    for (int i = tid; i < kJSlots * 32; i += NT) lut2[i] = S.pq32[i >> 5];
-    __syncthreads();
-}
-
-struct Row8 { float x[8]; float I[8]; };
-struct Exact8 { int J[8]; double emin; int sigma; };
-
-// Double-precision decision (Eq. 8 as a plain double-precision loop states it, lanes of a group
-// combined by a shuffle tree) for the groups whose lanes pass need != 0; every lane of the warp
-// calls.  The interval of every weight is found by direct search of the breakpoint list.
-template <int LPG>
-__device__ __noinline__ Exact8 exact_groups(const FitTables* S, Row8 r, int need) {
-    Exact8 out;
-    double e0 = 0.0, e1 = 0.0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        int J = 0;
-        if (need) {
-#pragma unroll 1
-            for (int i = 0; i < kNBP; ++i) J += (S->bp[i] < r.x[j]);
-            const double2 pq = S->PQ[J];
-            const double xd = (double)r.x[j], id = (double)r.I[j];
-            const double d0 = __dsub_rn(xd, pq.x), d1 = __dsub_rn(xd, pq.y);
-            e0 = __dadd_rn(e0, __dmul_rn(id, __dmul_rn(d0, d0)));
-            e1 = __dadd_rn(e1, __dmul_rn(id, __dmul_rn(d1, d1)));
-        }
-        out.J[j] = J;
-    }
-#pragma unroll
-    for (int s = LPG / 2; s; s >>= 1) {
-        e0 = __dadd_rn(e0, __shfl_xor_sync(0xFFFFFFFFu, e0, s));
-        e1 = __dadd_rn(e1, __shfl_xor_sync(0xFFFFFFFFu, e1, s));
-    }
-    out.sigma = e1 < e0;
-    out.emin = out.sigma ? e1 : e0;
-    return out;
-}
 
 constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
 

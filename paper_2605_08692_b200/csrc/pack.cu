@@ -1,413 +1,287 @@
 // The final pack pass (Algorithm 1 lines 17-20): BF16 tables, exact selection, 4-bit codes.
 //
-// For every weight it forms w~ = fl32(w * r) (Eq. 2), finds the interval J of the merged
-// breakpoint list of both tables that holds w~, and from J the nearest entry of T0 and of T1
-// (Eq. 4).  Per group it sums the two activation-weighted errors (Eq. 8), picks sigma, writes
-// the 4-bit codes under the chosen table (Eq. 6) and sigma into the sign bit of the scale.
-// (The template keeps a FIT variant of the same loop, which the fit rounds no longer use; the
-// round kernel lives in fit.cu.)
+// The tables are rounded to BF16 (RNE of the FP32 values) and sorted.  For every weight the pass
+// forms w~ = fl32(w * r) (Eq. 2) and finds, with the lookup tables of lookup.cuh, the interval of
+// the merged breakpoint list that holds it and the nearest entries P, Q of T0, T1 (Eq. 4).  Per
+// group it sums the two activation-weighted errors (Eq. 8), picks sigma, writes the 4-bit index
+// under the chosen table (Eq. 6; the index rides in the low mantissa bits of the constants the
+// lookup returns) and sigma into the sign bit of the scale.
 //
-// Merged breakpoints.  With sorted tables the nearest entry of table r is
-// #{i : w~ > mid_r,i}, mid_r,i = (T_r[i] + T_r[i+1]) / 2, and for a float x and a real m,
-// x > m  <=>  x > round_down_fp32(m).  The 30 rounded midpoints of both tables are sorted into
-// bp[0..29]; J(x) = #{j : bp[j] < x} in 0..30 determines both indices.  J is found from a
-// 1025-entry byte table over uniform bins of width 1/64 on (-8, 8) giving the number of
-// breakpoints below the bin's lower edge, followed by compares against the next breakpoints.
+// Exactness.  The group errors are summed in FP32 with constants that differ from the entries by
+// at most 2^-19 max|T|; groups inside the resulting error bound (see fit.cu) are re-evaluated in
+// double with the exact entries, so sigma equals the double-precision decision.  The interval
+// search itself is exact (rounded-down midpoints), hence so are the codes.
 //
-// Exactness of sigma.  The FP32 group errors decide sigma unless |E1 - E0| <= 2^-14 (E0 + E1);
-// such groups are re-evaluated in double in index order with the same operations a plain
-// double-precision loop uses, so sigma equals the double-precision decision.
+// Also reported: the Eq. 8 objective under the BF16 tables, sum_k I_k (w - w^)^2 in weight units,
+// the number of groups with E0 == E1 exactly (among those re-evaluated), of weights exactly
+// half-way between two different entries of their table, and of groups re-evaluated in double.
 //
-// Thread mapping.  A block works on items of 32 rows x 256 columns; each of its 8 warps takes
-// 4 rows, each lane 8 adjacent columns (one 128-bit load per row).  A group is 2 lanes
-// (g = 16) or 16 lanes (g = 128); group sums are xor-shuffle reductions.
-#include "internal.cuh"
+// Thread mapping as in the fit rounds: a block of NW warps takes items of 4 NW rows x 256 columns
+// in contiguous ranges, a warp 4 rows, a lane 8 adjacent columns (one 128-bit load per row, one
+// 32-bit store of 8 codes); the next item's rows are loaded while the current one is processed.
+// Error sums go through one partial per block, added in block order by the last block to finish.
+#include "lookup.cuh"
 
 namespace aaac {
 
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kRowsPerWarp = 4;
-constexpr int kRowsPerItem = kWarps * kRowsPerWarp;
-constexpr int kNBins = 1025;
-constexpr float kMagic = 12582912.f + 512.f;      // 1.5 * 2^23 + 512
-constexpr int kMagicBits = 0x4B400000;            // bits of 1.5 * 2^23
+constexpr int kPackWarps = 12;
+constexpr int kPackRep = 16;          // one copy of the {J_low, thr} table per lane of a half-warp: no conflicts
 
-struct Luts {
-    double Td[2 * kM];
-    float bp[32];                 // sorted breakpoints, bp[30] = bp[31] = +inf
-    float P[32], Q[32];           // nearest entry of T0 / T1 on interval J
-    float rlut[128];              // NVFP4: fl32(1 / s_eff) per E4M3 code
-    float slut[128];              // NVFP4: s_eff per E4M3 code
-    float tmp_b[32];
-    uint8_t tmp_src[32], tmp_exact[32];
-    uint8_t src[32], exact[32];   // table of origin; breakpoint is an exact midpoint of two different entries
-    uint8_t idx0[32], idx1[32];   // canonical (lowest duplicate) entry index on interval J
-    uint8_t clut[kNBins + 3];
-    double wsum[kWarps][kPartStride];
-    double tot[kPartStride];
-    int is_last;
-};
-
-struct Params {
+struct PackParams {
     const uint16_t* W;
     int64_t N, K, ldw;
-    const void* scales_in;        // FIT: positive scales (NVFP4 bytes); PACK: scales in/out
-    void* scales_out;
-    const float* rinv;            // FIT INT4
+    void* scales;                 // in: positive scales; out: sign bit = sigma
     const float* I;
-    const float* tensor_scale;    // PACK NVFP4
+    const float* tensor_scale;    // NVFP4
     Ctrl* ctrl;
     double* part;
-    double* err_slot;
-    const float* T01_f32;         // PACK
+    const float* T01_f32;
     uint16_t* T01_bf16;
     uint8_t* codes;
-    int64_t items;
-    int slabs;
+    int items, per_block, nrb;
 };
 
-__device__ __forceinline__ void sort16(double* t) {
-    for (int i = 1; i < kM; ++i) {
-        double v = t[i];
-        int j = i - 1;
-        while (j >= 0 && t[j] > v) { t[j + 1] = t[j]; --j; }
-        t[j + 1] = v;
-    }
-}
-
-template <int MODE, bool PACK>
-__device__ void build_luts(Luts& L, const Params& p) {
-    const int tid = threadIdx.x;
-    if (tid < 2 * kM) {
-        if (PACK) {
-            const uint32_t b = f32_to_bf16_rne(p.T01_f32[tid]);
-            L.Td[tid] = (double)__uint_as_float(b << 16);
-        } else {
-            L.Td[tid] = p.ctrl->T[tid];
-        }
-    }
-    __syncthreads();
-    if (PACK && tid < 2) sort16(L.Td + tid * kM);
-    __syncthreads();
-    if (PACK && blockIdx.x == 0 && tid < 2 * kM) p.T01_bf16[tid] = (uint16_t)(__float_as_uint((float)L.Td[tid]) >> 16);
-    if (tid < kNBP) {
-        const int r = tid / 15, i = tid % 15;
-        const double a = L.Td[r * kM + i], b = L.Td[r * kM + i + 1];
-        const double mid = (a + b) * 0.5;
-        const float f = f32_round_down(mid);
-        L.tmp_b[tid] = f;
-        L.tmp_src[tid] = (uint8_t)r;
-        L.tmp_exact[tid] = (uint8_t)(((double)f == mid) && (a != b));
-    }
-    if (tid >= 30 && tid < 32) L.bp[tid] = __int_as_float(0x7F800000);
-    __syncthreads();
-    if (tid < kNBP) {
-        const float b = L.tmp_b[tid];
-        int rank = 0;
-        for (int j = 0; j < kNBP; ++j) rank += (L.tmp_b[j] < b) || (L.tmp_b[j] == b && j < tid);
-        L.bp[rank] = b;
-        L.src[rank] = L.tmp_src[tid];
-        L.exact[rank] = L.tmp_exact[tid];
-    }
-    if (MODE == AAAC_NVFP4 && tid >= 128 && tid < 256) {
-        const int c = tid - 128;
-        const float s_t = PACK ? p.tensor_scale[0] : p.ctrl->s_t;
-        const float s = __fmul_rn(e4m3_value((uint32_t)c), s_t);
-        L.slut[c] = s;
-        L.rlut[c] = c ? __frcp_rn(s) : 0.f;
-    }
-    __syncthreads();
-    if (tid < kNJ) {
-        int i0 = 0, i1 = 0;
-        for (int j = 0; j < tid; ++j) { i0 += (L.src[j] == 0); i1 += (L.src[j] == 1); }
-        while (i0 > 0 && L.Td[i0 - 1] == L.Td[i0]) --i0;
-        while (i1 > 0 && L.Td[kM + i1 - 1] == L.Td[kM + i1]) --i1;
-        L.idx0[tid] = (uint8_t)i0;
-        L.idx1[tid] = (uint8_t)i1;
-        L.P[tid] = (float)L.Td[i0];
-        L.Q[tid] = (float)L.Td[kM + i1];
-    }
-    for (int b = tid; b < kNBins; b += kThreads) {
-        const float edge = ((float)b - 512.5f) * 0.015625f;    // lower edge of the bin, exact
-        int c = 0;
-        for (int j = 0; j < kNBP; ++j) c += (L.bp[j] < edge);
-        L.clut[b] = (uint8_t)c;
-    }
-    __syncthreads();
-}
-
-// index of the nearest entry in double, lowest index on ties
-__device__ __forceinline__ int nearest_d(const double* T, double x) {
-    int best = 0;
-    double bd = fabs(__dsub_rn(x, T[0]));
-#pragma unroll 1
-    for (int i = 1; i < kM; ++i) {
-        const double d = fabs(__dsub_rn(x, T[i]));
-        if (d < bd) { bd = d; best = i; }
-    }
-    return best;
-}
-
-// Double-precision evaluation of Eq. 8 for the groups whose lanes have need != 0.  Terms are
-// I * (d * d) with d = w~ - T[nearest], added in index order.  Every lane of the warp calls this.
-template <int LPG>
-__device__ void exact_groups(const Luts& L, const float (&x)[8], const float (&Iv)[8], int lane, bool need,
-                             bool& sigma, double& emin, bool& tie) {
-    unsigned mask = __ballot_sync(0xFFFFFFFFu, need);
-    while (mask) {
-        const int gbase = (__ffs(mask) - 1) & ~(LPG - 1);
-        const bool mine = (lane & ~(LPG - 1)) == gbase;
-        double t0[8], t1[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            t0[j] = 0.0;
-            t1[j] = 0.0;
-            if (mine) {
-                const double xd = (double)x[j], id = (double)Iv[j];
-                const double d0 = __dsub_rn(xd, L.Td[nearest_d(L.Td, xd)]);
-                const double d1 = __dsub_rn(xd, L.Td[kM + nearest_d(L.Td + kM, xd)]);
-                t0[j] = __dmul_rn(id, __dmul_rn(d0, d0));
-                t1[j] = __dmul_rn(id, __dmul_rn(d1, d1));
-            }
-        }
-        double E0 = 0.0, E1 = 0.0;
-        for (int l = 0; l < LPG; ++l) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                E0 = __dadd_rn(E0, __shfl_sync(0xFFFFFFFFu, t0[j], gbase + l));
-                E1 = __dadd_rn(E1, __shfl_sync(0xFFFFFFFFu, t1[j], gbase + l));
-            }
-        }
-        if (mine) {
-            sigma = E1 < E0;
-            emin = sigma ? E1 : E0;
-            tie = (E0 == E1);
-        }
-        mask &= ~(((LPG == 32) ? 0xFFFFFFFFu : ((1u << LPG) - 1u)) << gbase);
-    }
-}
-
-template <int MODE, bool PACK>
-__global__ void __launch_bounds__(kThreads, 1) fit_kernel(const Params p) {
+template <int MODE, int NW, int REP>
+__global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;
-    extern __shared__ __align__(16) unsigned char dyn_smem[];
-    __shared__ Luts L;
+    constexpr int R = kRowsPerWarp;
+    constexpr int kRowsPerItem = R * NW;
+    constexpr int kLut1Bytes = REP * kNBins * 8;
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ FitTables S;
+    __shared__ float slut[128];                      // NVFP4: s_eff per E4M3 code
+    __shared__ double wsum[NW][2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    build_luts<MODE, PACK>(L, p);
-
-    float2* bins = reinterpret_cast<float2*>(dyn_smem) + (size_t)warp * (2 * kNJ * 32) + lane;
-    if (!PACK) {
-        for (int b = 0; b < 2 * kNJ; ++b) bins[b * 32] = make_float2(0.f, 0.f);
+    // ---- BF16 tables (Algorithm 1 line 17), sorted
+    float tb = 0.f;
+    if (tid < 2 * kM) {
+        tb = __uint_as_float(f32_to_bf16_rne(p.T01_f32[tid]) << 16);
+        S.tot[tid] = (double)tb;
     }
+    if (MODE == AAAC_NVFP4 && tid >= 64 && tid < 192) {
+        const int c = tid - 64;
+        const float sv = __fmul_rn(e4m3_value((uint32_t)c), p.tensor_scale[0]);
+        slut[c] = sv;
+        S.rlut[c] = c ? __frcp_rn(sv) : 0.f;
+    }
+    __syncthreads();
+    if (tid < 2 * kM) {
+        const int r = tid & 16;
+        int rank = 0;
+        for (int i = 0; i < kM; ++i) {
+            const double ti = S.tot[r + i];
+            rank += (ti < (double)tb) || (ti == (double)tb && i < (tid & 15));
+        }
+        S.Td[r + rank] = (double)tb;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0 && tid < 2 * kM) p.T01_bf16[tid] = (uint16_t)(__float_as_uint((float)S.Td[tid]) >> 16);
+    build_tables<MODE, NW, REP>(S, dyn);
+
+    const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
+    const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;
+    const int c0 = (int)(sm_base + kLut1Bytes + lane * 8), c1 = c0 + kSlotBytes;
+    constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
+    constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
+    const float tmax283 = S.tmax283;
+
     double Eacc = 0.0, Eout = 0.0;
     uint32_t n_sig_tie = 0, n_idx_tie = 0, n_exact = 0;
-    const int64_t Gr = p.K / G;
 
-    for (int64_t item = blockIdx.x; item < p.items; item += gridDim.x) {
-        const int slab = (int)(item % p.slabs);
-        const int64_t row0 = (item / p.slabs) * kRowsPerItem + warp * kRowsPerWarp;
-        const int64_t col0 = (int64_t)slab * 256 + lane * 8;
-        const bool col_ok = col0 < p.K;
-        float Iv[8];
-        if (col_ok) {
-            const float4 a = __ldg(reinterpret_cast<const float4*>(p.I + col0));
-            const float4 b = __ldg(reinterpret_cast<const float4*>(p.I + col0 + 4));
-            Iv[0] = a.x; Iv[1] = a.y; Iv[2] = a.z; Iv[3] = a.w;
-            Iv[4] = b.x; Iv[5] = b.y; Iv[6] = b.z; Iv[7] = b.w;
-        } else {
+    const int N = (int)p.N, K = (int)p.K;
+    const int Gr = K / G;
+    const int it0 = blockIdx.x * p.per_block;
+    const int it1 = min(p.items, it0 + p.per_block);
+
+    uint4 nv[R];
+    uint32_t ns[R];           // scale bits (sign clear): E4M3 byte or BF16 pattern
+    auto load_item = [&](int slab, int rb) {
+        const int col0 = slab * 256 + lane * 8;
+        const int row0 = rb * kRowsPerItem + warp * R;
+        const uint16_t* wp = p.W + (size_t)row0 * (size_t)p.ldw + col0;
+        const uint32_t g0 = (uint32_t)col0 / G;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
-        }
-        uint4 v[kRowsPerWarp];
-        float rinv[kRowsPerWarp], sval[kRowsPerWarp];
-        uint32_t sbits[kRowsPerWarp];
-#pragma unroll
-        for (int u = 0; u < kRowsPerWarp; ++u) {
-            const int64_t row = row0 + u;
-            const bool ok = col_ok && row < p.N;
-            v[u] = make_uint4(0, 0, 0, 0);
-            rinv[u] = 0.f;
-            sval[u] = 0.f;
-            sbits[u] = 0;
-            if (ok) {
-                v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + row * p.ldw + col0));
-                const int64_t gi = row * Gr + col0 / G;
-                if (MODE == AAAC_NVFP4) {
-                    sbits[u] = reinterpret_cast<const uint8_t*>(p.scales_in)[gi] & 0x7Fu;
-                } else if (PACK) {
-                    sbits[u] = reinterpret_cast<const uint16_t*>(p.scales_in)[gi] & 0x7FFFu;
-                } else {
-                    rinv[u] = __ldg(p.rinv + gi);
-                }
+        for (int u = 0; u < R; ++u) {
+            const int row = row0 + u;
+            nv[u] = make_uint4(0, 0, 0, 0);
+            ns[u] = 0u;
+            if (col0 < K && row < N) {
+                nv[u] = __ldcs(reinterpret_cast<const uint4*>(wp + (size_t)u * (size_t)p.ldw));
+                const size_t gi = (size_t)row * (size_t)Gr + g0;
+                if (MODE == AAAC_NVFP4) ns[u] = reinterpret_cast<const uint8_t*>(p.scales)[gi];
+                else ns[u] = reinterpret_cast<const uint16_t*>(p.scales)[gi];
             }
         }
+    };
+
+    int cur_slab = -1;
+    float Iv[8];
+    float isum = 0.f;
+    bool col_ok = false;
 #pragma unroll
-        for (int u = 0; u < kRowsPerWarp; ++u) {
-            const int64_t row = row0 + u;
-            const bool ok = col_ok && row < p.N;
+    for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
+
+    int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
+    int nslab = slab, nrb = rb;
+    if (it0 < it1) load_item(slab, rb);
+    for (int item = it0; item < it1; ++item) {
+        uint4 v[R];
+        uint32_t sc[R];
+#pragma unroll
+        for (int u = 0; u < R; ++u) { v[u] = nv[u]; sc[u] = ns[u]; }
+        slab = nslab;
+        rb = nrb;
+        if (++nrb == p.nrb) { nrb = 0; ++nslab; }
+        if (item + 1 < it1) load_item(nslab, nrb);
+
+        const int col0 = slab * 256 + lane * 8;
+        if (slab != cur_slab) {
+            cur_slab = slab;
+            col_ok = col0 < K;
+            isum = 0.f;
+            if (col_ok) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(p.I + col0));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(p.I + col0 + 4));
+                Iv[0] = a.x; Iv[1] = a.y; Iv[2] = a.z; Iv[3] = a.w;
+                Iv[4] = b.x; Iv[5] = b.y; Iv[6] = b.z; Iv[7] = b.w;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) isum += Iv[j];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
+            }
+#pragma unroll
+            for (int o = LPG / 2; o; o >>= 1) isum += __shfl_xor_sync(0xFFFFFFFFu, isum, o);
+            isum *= 1.0001f;
+        }
+        const int row0 = rb * kRowsPerItem + warp * R;
+
+#pragma unroll
+        for (int u = 0; u < R; ++u) {
+            const int row = row0 + u;
+            if (row >= N) break;                            // uniform over the warp
+            const uint32_t sbits = MODE == AAAC_NVFP4 ? (sc[u] & 0x7Fu) : (sc[u] & 0x7FFFu);
+            float sval, rinv;
             if (MODE == AAAC_NVFP4) {
-                rinv[u] = L.rlut[sbits[u]];
-                sval[u] = L.slut[sbits[u]];
-            } else if (PACK) {
-                sval[u] = __uint_as_float(sbits[u] << 16);
-                rinv[u] = ok ? __frcp_rn(sval[u]) : 0.f;
+                sval = slut[sbits];
+                rinv = S.rlut[sbits];
+            } else {
+                sval = __uint_as_float(sbits << 16);
+                rinv = col_ok ? __frcp_rn(sval) : 0.f;
             }
             const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
             float x[8];
-            int J[8];
+            float2 pq[8];
+            bool tcand = false;                             // some w~ equals the breakpoint of its bin
             float e0 = 0.f, e1 = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
-                x[j] = __fmul_rn(wf, rinv[u]);
-                int bin = __float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) - kMagicBits;
-                bin = min(max(bin, 0), kNBins - 1);
-                int Jj = L.clut[bin];
-                while (x[j] > L.bp[Jj]) ++Jj;
-                J[j] = Jj;
-                const float d0 = x[j] - L.P[Jj], d1 = x[j] - L.Q[Jj];
-                e0 = __fmaf_rn(__fmul_rn(Iv[j], d0), d0, e0);
-                e1 = __fmaf_rn(__fmul_rn(Iv[j], d1), d1, e1);
+                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
+                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) & kBinMask;
+                const uint2 e = lds_table_u2(lut1_lane + off);
+                const float thr = __uint_as_float(e.y);
+                tcand |= (x[j] == thr);
+                pq[j] = lds_table_f2(e.x + (uint32_t)((x[j] > thr) ? c1 : c0));
+                const float u0 = __fsub_rn(x[j], pq[j].x), u1 = __fsub_rn(x[j], pq[j].y);
+                e0 = __fmaf_rn(__fmul_rn(Iv[j], u0), u0, e0);
+                e1 = __fmaf_rn(__fmul_rn(Iv[j], u1), u1, e1);
             }
 #pragma unroll
-            for (int o = LPG / 2; o; o >>= 1) {
-                e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, o);
-                e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, o);
+            for (int s = LPG / 2; s; s >>= 1) {
+                e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, s);
+                e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, s);
             }
-            bool sigma = e1 < e0;
-            double emin = (double)(sigma ? e1 : e0);
-            bool tie = false;
-            const bool near = ok && (fabsf(e1 - e0) <= 0x1p-14f * (e0 + e1));
+            const float es = e0 + e1;
+            const float tau = 0x1p-24f * __fmaf_rn(tmax283, __fsqrt_ru(__fmul_ru(isum, es)), 16.f * es);
+            const bool near = !(fabsf(e1 - e0) > tau) && (col_ok || !(es == es));
+            bool sg = e1 < e0;
+            double emin = (double)(sg ? e1 : e0);
             if (__any_sync(0xFFFFFFFFu, near)) {
-                exact_groups<LPG>(L, x, Iv, lane, near, sigma, emin, tie);
-                if (near && (lane % LPG) == 0) { ++n_exact; n_sig_tie += tie; }
+                Row8 r;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = Iv[j]; }
+                const Exact8 ex = exact_groups<LPG>(&S, r, (int)near);
+                if (near) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) pq[j] = lds_table_f2((uint32_t)(c0 + ex.J[j] * kSlotBytes));
+                    sg = ex.sigma != 0;
+                    emin = ex.emin;
+                    tcand = true;                           // poisoned slots carry no breakpoint to compare with
+                    if (col_ok && (lane % LPG) == 0) { ++n_exact; n_sig_tie += ex.tie; }
+                }
             }
-            if (ok && (lane % LPG) == 0) Eacc += emin;
-
-            if (!PACK) {
-                if (ok) {
-                    float2* b = bins + (sigma ? kNJ * 32 : 0);
+            if (!col_ok) continue;
+            if ((lane % LPG) == 0) Eacc += emin;
+            // codes (Eq. 6) and the error in weight units
+            uint32_t word = 0;
+            float eo = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float2 a = b[J[j] * 32];
-                        a.x = __fmaf_rn(Iv[j], x[j], a.x);
-                        a.y += Iv[j];
-                        b[J[j] * 32] = a;
-                    }
-                }
-            } else if (ok) {
-                uint32_t word = 0;
-                float eo = 0.f;
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t cb = __float_as_uint(sg ? pq[j].y : pq[j].x);
+                word |= (cb & kIdxMask) << (4 * j);
+                const float tv = __uint_as_float(cb & ~kIdxMask);          // the BF16 entry itself
+                const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
+                const float dw = __fmaf_rn(-tv, sval, wf);
+                eo = __fmaf_rn(__fmul_rn(Iv[j], dw), dw, eo);
+            }
+            Eout += (double)eo;
+            if (tcand) {
+                // weights exactly half-way between two different entries of the chosen table
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int Jj = J[j];
-                    const uint32_t idx = sigma ? L.idx1[Jj] : L.idx0[Jj];
-                    word |= idx << (4 * j);
-                    const float tv = sigma ? L.Q[Jj] : L.P[Jj];
-                    const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
-                    const float dw = __fmaf_rn(-tv, sval[u], wf);
-                    eo = __fmaf_rn(__fmul_rn(Iv[j], dw), dw, eo);
-                    for (int jj = Jj; jj < kNBP && L.bp[jj] == x[j]; ++jj)
-                        if (L.src[jj] == (uint8_t)sigma && L.exact[jj]) { ++n_idx_tie; break; }
-                }
-                Eout += (double)eo;
-                *reinterpret_cast<uint32_t*>(p.codes + ((row * p.K + col0) >> 1)) = word;
-                if ((lane % LPG) == 0) {
-                    const int64_t gi = row * Gr + col0 / G;
-                    if (MODE == AAAC_NVFP4)
-                        reinterpret_cast<uint8_t*>(p.scales_out)[gi] = (uint8_t)(sbits[u] | (sigma ? 0x80u : 0u));
-                    else
-                        reinterpret_cast<uint16_t*>(p.scales_out)[gi] = (uint16_t)(sbits[u] | (sigma ? 0x8000u : 0u));
-                }
+                for (int j = 0; j < 8; ++j)
+                    for (int jj = 0; jj < kNBP; ++jj)
+                        if (S.bp[jj] == x[j] && S.src[jj] == (uint8_t)sg && S.exact[jj]) { ++n_idx_tie; break; }
+            }
+            *reinterpret_cast<uint32_t*>(p.codes + (((size_t)row * (size_t)K + col0) >> 1)) = word;
+            if ((lane % LPG) == 0) {
+                const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+                if (MODE == AAAC_NVFP4)
+                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
+                else
+                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits | (sg ? 0x8000u : 0u));
             }
         }
     }
 
-    // ---- block partial ----
-    if (!PACK) {
-        __syncwarp();
-        for (int b = 0; b < 2 * kNJ; ++b) {
-            const float2 a = bins[b * 32];
-            double sx = (double)a.x, sy = (double)a.y;
+    // ---- block partial of the two error sums; integer statistics by atomics ----
 #pragma unroll
-            for (int o = 16; o; o >>= 1) {
-                sx += __shfl_xor_sync(0xFFFFFFFFu, sx, o);
-                sy += __shfl_xor_sync(0xFFFFFFFFu, sy, o);
-            }
-            if (lane == 0) { L.wsum[warp][b] = sx; L.wsum[warp][2 * kNJ + b] = sy; }
-        }
+    for (int s = 16; s; s >>= 1) {
+        Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, s);
+        Eout += __shfl_xor_sync(0xFFFFFFFFu, Eout, s);
+        n_sig_tie += __shfl_xor_sync(0xFFFFFFFFu, n_sig_tie, s);
+        n_idx_tie += __shfl_xor_sync(0xFFFFFFFFu, n_idx_tie, s);
+        n_exact += __shfl_xor_sync(0xFFFFFFFFu, n_exact, s);
     }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, o);
-        Eout += __shfl_xor_sync(0xFFFFFFFFu, Eout, o);
-    }
-    if (lane == 0) { L.wsum[warp][4 * kNJ] = Eacc; L.wsum[warp][4 * kNJ + 1] = Eout; }
-    if (PACK) {
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            n_sig_tie += __shfl_xor_sync(0xFFFFFFFFu, n_sig_tie, o);
-            n_idx_tie += __shfl_xor_sync(0xFFFFFFFFu, n_idx_tie, o);
-            n_exact += __shfl_xor_sync(0xFFFFFFFFu, n_exact, o);
-        }
-        if (lane == 0) {
-            if (n_sig_tie) atomicAdd(&p.ctrl->pack_stats[0], (unsigned long long)n_sig_tie);
-            if (n_idx_tie) atomicAdd(&p.ctrl->pack_stats[1], (unsigned long long)n_idx_tie);
-            if (n_exact) atomicAdd(&p.ctrl->pack_stats[2], (unsigned long long)n_exact);
-        }
+    if (lane == 0) {
+        wsum[warp][0] = Eacc;
+        wsum[warp][1] = Eout;
+        if (n_sig_tie) atomicAdd(&p.ctrl->pack_stats[0], (unsigned long long)n_sig_tie);
+        if (n_idx_tie) atomicAdd(&p.ctrl->pack_stats[1], (unsigned long long)n_idx_tie);
+        if (n_exact) atomicAdd(&p.ctrl->pack_stats[2], (unsigned long long)n_exact);
     }
     __syncthreads();
-    constexpr int kUsed = 4 * kNJ + 2;
-    if (tid < kUsed) {
+    if (tid < 2) {
         double s = 0.0;
-        const int lo = PACK ? 4 * kNJ : 0;
-        if (tid >= lo) {
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) s += L.wsum[w][tid];
-        }
-        p.part[(int64_t)blockIdx.x * kPartStride + tid] = s;
+        for (int w = 0; w < NW; ++w) s += wsum[w][tid];
+        p.part[(size_t)blockIdx.x * kPartStride + tid] = s;
     }
     __threadfence();
     __syncthreads();
-    if (tid == 0) L.is_last = (atomicAdd(&p.ctrl->done, 1u) == gridDim.x - 1);
+    if (tid == 0) S.is_last = (atomicAdd(&p.ctrl->done, 1u) == gridDim.x - 1);
     __syncthreads();
-    if (!L.is_last) return;
-
-    // ---- last block: reduce all partials in block order, then update the tables ----
+    if (!S.is_last) return;
     __threadfence();
-    if (tid < kUsed) {
+    if (tid < 2) {
         double s = 0.0;
-        for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(p.part + (int64_t)b * kPartStride + tid);
-        L.tot[tid] = s;
+        for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(p.part + (size_t)b * kPartStride + tid);
+        p.ctrl->pack_err[tid] = s;
     }
-    __syncthreads();
-    if (tid == 0) {
-        if (!PACK) {
-            double S[2 * kM], Wt[2 * kM];
-            for (int i = 0; i < 2 * kM; ++i) { S[i] = 0.0; Wt[i] = 0.0; }
-            for (int r = 0; r < 2; ++r)
-                for (int j = 0; j < kNJ; ++j) {
-                    const int i = r * kM + (r ? L.idx1[j] : L.idx0[j]);
-                    S[i] += L.tot[r * kNJ + j];
-                    Wt[i] += L.tot[2 * kNJ + r * kNJ + j];
-                }
-            double Tn[2 * kM];
-            for (int i = 0; i < 2 * kM; ++i) Tn[i] = (Wt[i] > 0.0) ? __ddiv_rn(S[i], Wt[i]) : L.Td[i];
-            sort16(Tn);
-            sort16(Tn + kM);
-            for (int i = 0; i < 2 * kM; ++i) p.ctrl->T[i] = Tn[i];
-            if (p.err_slot) *p.err_slot = L.tot[4 * kNJ];
-        } else {
-            p.ctrl->pack_err[0] = L.tot[4 * kNJ];
-            p.ctrl->pack_err[1] = L.tot[4 * kNJ + 1];
-        }
-        p.ctrl->done = 0;
-    }
+    if (tid == 0) p.ctrl->done = 0;
 }
 
 __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long long* stats) {
@@ -418,24 +292,38 @@ __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long lo
     }
 }
 
+template <int MODE>
+cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t st) {
+    constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kJSlots * kSlotBytes;
+    auto kern = pack_kernel<MODE, kPackWarps, kPackRep>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kPackWarps * 32, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,
                         const float* T01_f32, uint16_t* T01_bf16, void* scales, const float* tensor_scale,
                         uint8_t* codes, double* err_out, unsigned long long* stats, const Workspace& ws,
                         cudaStream_t st) {
-    Params p{};
+    PackParams p{};
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
-    p.scales_in = scales; p.scales_out = scales; p.I = I; p.tensor_scale = tensor_scale;
+    p.scales = scales; p.I = I; p.tensor_scale = tensor_scale;
     p.ctrl = ws.ctrl; p.part = ws.part; p.T01_f32 = T01_f32; p.T01_bf16 = T01_bf16; p.codes = codes;
-    p.slabs = (int)((K + 255) / 256);
-    p.items = (int64_t)p.slabs * ((N + kRowsPerItem - 1) / kRowsPerItem);
-    int64_t grid = (int64_t)sm_count() * 2;
-    if (grid > p.items) grid = p.items;
+    const int64_t slabs = (K + 255) / 256;
+    constexpr int kRowsPerItem = kRowsPerWarp * kPackWarps;
+    const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
+    if (N > 0x7FFFFFFF || K > 0x7FFFFFFF || items > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    int64_t grid = sm_count();
+    if (grid > items) grid = items;
     if (grid > kMaxBlocks) grid = kMaxBlocks;
-    if (mode == AAAC_INT4) fit_kernel<AAAC_INT4, true><<<(unsigned)grid, kThreads, 0, st>>>(p);
-    else fit_kernel<AAAC_NVFP4, true><<<(unsigned)grid, kThreads, 0, st>>>(p);
-    cudaError_t e = cudaGetLastError();
+    const int64_t per_block = (items + grid - 1) / grid;
+    grid = (items + per_block - 1) / per_block;
+    p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
+    cudaError_t e = mode == AAAC_INT4 ? launch_pack_variant<AAAC_INT4>(p, (unsigned)grid, st)
+                                      : launch_pack_variant<AAAC_NVFP4>(p, (unsigned)grid, st);
     if (e != cudaSuccess) return e;
     export_pack_kernel<<<1, 32, 0, st>>>(ws.ctrl, err_out, stats);
     return cudaGetLastError();
