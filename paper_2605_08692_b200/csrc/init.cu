@@ -8,7 +8,9 @@
 //   2. one block turns the histogram into a prefix sum, finds the bin and the rank inside the
 //      bin of every requested order statistic, and gives each distinct bin a slot;
 //   3. a second pass over W appends the (order-preserving integer keys of the) values that fall
-//      into a slotted bin to that slot's list -- the lists' sizes are known from step 1;
+//      into a slotted bin to that slot's list -- the lists' sizes are known from step 1.  A block
+//      stages its candidates in shared memory and reserves list space once per slot, so the
+//      global counters see one atomic per block and slot instead of one per candidate;
 //   4. one block per slot selects the requested ranks of its list by an 8-bit radix select;
 //   5. the table entries are interpolated in double and rounded to FP32.
 // Integer atomics only, so the result does not depend on scheduling.
@@ -44,53 +46,121 @@ __device__ __forceinline__ float group_rinv(const void* scales, int64_t gi, floa
     return __frcp_rn(__fmul_rn(e4m3_value(c), s_t));
 }
 
-// PASS 0: histogram.  PASS 1: collect candidates of slotted bins.
-template <int MODE, int PASS>
+// Step 1: histogram of every w~ (shared-memory counters per block, merged with integer atomics).
+// A warp takes two 256-column pieces per iteration so that two loads are in flight.
+template <int MODE>
 __global__ void __launch_bounds__(256)
-quantile_scan_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
-                     const void* __restrict__ scales, Ctrl* ctrl, uint32_t* __restrict__ hist,
-                     const uint8_t* __restrict__ slot_of_bin, uint32_t* __restrict__ list) {
+quantile_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
+                     const void* __restrict__ scales, const Ctrl* ctrl, uint32_t* __restrict__ hist) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
-    extern __shared__ uint32_t sm[];                 // PASS 0: kQBins counters; PASS 1: kQBins/4 words of slot ids
+    extern __shared__ uint32_t sm[];                      // kQBins counters
     const int lane = threadIdx.x & 31;
-    if (PASS == 0) {
-        for (int i = threadIdx.x; i < kQBins; i += blockDim.x) sm[i] = 0;
-    } else {
+    for (int i = threadIdx.x; i < kQBins; i += blockDim.x) sm[i] = 0;
+    __syncthreads();
+    const float s_t = ctrl->s_t;
+    const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t it = warp0; it < items; it += 2 * nwarps) {
+        uint4 v[2];
+        float r[2];
+        bool ok[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t i2 = it + h * nwarps;
+            const int64_t row = i2 / slabs, col = (i2 % slabs) * 256 + lane * 8;
+            ok[h] = i2 < items && col < K;
+            v[h] = make_uint4(0, 0, 0, 0);
+            r[h] = 0.f;
+            if (ok[h]) {
+                v[h] = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
+                r[h] = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            if (!ok[h]) continue;
+            const uint32_t w[4] = {v[h].x, v[h].y, v[h].z, v[h].w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                atomicAdd(&sm[qbin(__fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r[h]))], 1u);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kQBins; i += blockDim.x)
+        if (sm[i]) atomicAdd(&hist[i], sm[i]);
+}
+
+// Step 3: candidates of the slotted bins, staged per block.
+constexpr int kStageCap = 4096;                  // staged candidates per block
+constexpr int kStageRoom = 256 * 8;              // most candidates one block iteration can add
+
+template <int MODE>
+__global__ void __launch_bounds__(256)
+quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
+                        const void* __restrict__ scales, Ctrl* ctrl, const uint8_t* __restrict__ slot_of_bin,
+                        uint32_t* __restrict__ list) {
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
+    extern __shared__ uint32_t sm[];                      // kQBins bytes of slot ids
+    __shared__ uint32_t buf_key[kStageCap];
+    __shared__ uint8_t buf_slot[kStageCap];
+    __shared__ uint16_t buf_pos[kStageCap];
+    __shared__ uint32_t cnt[kQReq];
+    __shared__ unsigned long long base[kQReq];
+    __shared__ uint32_t nbuf;
+    const int tid = threadIdx.x, lane = tid & 31;
+    {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(slot_of_bin);
-        for (int i = threadIdx.x; i < kQBins / 4; i += blockDim.x) sm[i] = src[i];
+        for (int i = tid; i < kQBins / 4; i += blockDim.x) sm[i] = src[i];
+        if (tid == 0) nbuf = 0;
     }
     __syncthreads();
     const uint8_t* sm_slot = reinterpret_cast<const uint8_t*>(sm);
     const float s_t = ctrl->s_t;
     const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
-    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + tid) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    for (int64_t it = warp0; it < items; it += nwarps) {
-        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
-        if (col >= K) continue;
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
-        const float r = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const int64_t iters = (items + nwarps - 1) / nwarps;
+
+    auto flush = [&]() {                                  // called by the whole block
+        const uint32_t n = nbuf;
+        if (tid < kQReq) cnt[tid] = 0;
+        __syncthreads();
+        for (uint32_t i = tid; i < n; i += blockDim.x) buf_pos[i] = (uint16_t)atomicAdd(&cnt[buf_slot[i]], 1u);
+        __syncthreads();
+        if (tid < kQReq && cnt[tid])
+            base[tid] = ctrl->slot_off[tid] + atomicAdd(&ctrl->slot_fill[tid], cnt[tid]);
+        __syncthreads();
+        for (uint32_t i = tid; i < n; i += blockDim.x) list[base[buf_slot[i]] + buf_pos[i]] = buf_key[i];
+        __syncthreads();
+        if (tid == 0) nbuf = 0;
+        __syncthreads();
+    };
+
+    for (int64_t k = 0; k < iters; ++k) {
+        const int64_t it = warp0 + k * nwarps;
+        if (it < items) {
+            const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
+            if (col < K) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
+                const float r = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
-            const int b = qbin(x);
-            if (PASS == 0) {
-                atomicAdd(&sm[b], 1u);
-            } else {
-                const uint32_t s = sm_slot[b];
-                if (s != 0xFFu) {
-                    const uint32_t pos = atomicAdd(&ctrl->slot_fill[s], 1u);
-                    list[ctrl->slot_off[s] + pos] = float_key(x);
+                for (int j = 0; j < 8; ++j) {
+                    const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
+                    const uint32_t s = sm_slot[qbin(x)];
+                    if (s != 0xFFu) {
+                        const uint32_t pos = atomicAdd(&nbuf, 1u);
+                        buf_key[pos] = float_key(x);
+                        buf_slot[pos] = (uint8_t)s;
+                    }
                 }
             }
         }
-    }
-    if (PASS == 0) {
         __syncthreads();
-        for (int i = threadIdx.x; i < kQBins; i += blockDim.x)
-            if (sm[i]) atomicAdd(&hist[i], sm[i]);
+        if (nbuf > kStageCap - kStageRoom) flush();       // uniform: nbuf is read after the barrier
     }
+    flush();
 }
 
 // one block of 1024 threads: prefix sum, bin + local rank of every request, slots
@@ -105,9 +175,29 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned lon
     for (int i = 0; i < per; ++i) s += hist[tid * per + i];
     chunk[tid] = s;
     __syncthreads();
-    if (tid == 0) {
-        unsigned long long run = 0;
-        for (int i = 0; i < 1024; ++i) { const unsigned long long c = chunk[i]; chunk[i] = run; run += c; }
+    // exclusive prefix of the 1024 chunk sums: warp scans, then a scan of the 32 warp totals
+    {
+        const int lane = tid & 31, warp = tid >> 5;
+        unsigned long long v = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+            if (lane >= o) v += t;
+        }
+        __shared__ unsigned long long wtot[32];
+        if (lane == 31) wtot[warp] = v;
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long w = wtot[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, w, o);
+                if (lane >= o) w += t;
+            }
+            wtot[lane] = w;                               // inclusive
+        }
+        __syncthreads();
+        chunk[tid] = v - s + (warp ? wtot[warp - 1] : 0ull);
     }
     __syncthreads();
     unsigned long long run = chunk[tid];
@@ -118,57 +208,106 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned lon
     }
     if (tid == 1023) prefix[kQBins] = run;
     __syncthreads();
+    __shared__ unsigned long long req_cnt[kQReq];
+    __shared__ int req_first[kQReq];
     if (tid < kQReq) {
+        // the bin that holds rank r: first the chunk (exclusive chunk prefixes are in shared
+        // memory), then a walk over the chunk's bins
         const unsigned long long r = ctrl->rank[tid];
-        int lo = 0, hi = kQBins;                          // last bin with prefix[bin] <= r
+        int lo = 0, hi = 1024;                            // last chunk with chunk[c] <= r
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (prefix[mid] <= r) lo = mid; else hi = mid;
+            if (chunk[mid] <= r) lo = mid; else hi = mid;
         }
-        req_bin[tid] = lo;
-        ctrl->req_local[tid] = r - prefix[lo];
+        unsigned long long base = chunk[lo];
+        int b = lo * per;
+        unsigned long long h = hist[b];
+        while (b < kQBins - 1 && r >= base + h) { base += h; ++b; h = hist[b]; }
+        req_bin[tid] = b;
+        req_cnt[tid] = h;
+        ctrl->req_local[tid] = r - base;
     }
     __syncthreads();
-    if (tid == 0) {
-        uint32_t ns = 0;
+    if (tid < kQReq) {
+        // a slot per distinct bin, in order of first appearance among the requests
+        int first = tid;
+        for (int q = 0; q < tid; ++q)
+            if (req_bin[q] == req_bin[tid]) { first = q; break; }
+        req_first[tid] = first;
+    }
+    __syncthreads();
+    if (tid < kQReq) {
+        uint32_t slot = 0;
         unsigned long long off = 0;
-        for (int q = 0; q < kQReq; ++q) {
-            const int b = req_bin[q];
-            if (slot_of_bin[b] == 0xFF) {
-                slot_of_bin[b] = (uint8_t)ns;
-                ctrl->slot_off[ns] = off;
-                ctrl->slot_fill[ns] = 0;
-                off += hist[b];
-                ++ns;
-            }
-            ctrl->req_slot[q] = slot_of_bin[b];
+        const int first = req_first[tid];
+        for (int q = 0; q < first; ++q)
+            if (req_first[q] == q) { ++slot; off += req_cnt[q]; }
+        ctrl->req_slot[tid] = slot;
+        if (first == tid) {
+            slot_of_bin[req_bin[tid]] = (uint8_t)slot;
+            ctrl->slot_off[slot] = off;
+            ctrl->slot_fill[slot] = 0;
         }
-        ctrl->slot_off[ns] = off;
-        ctrl->nslots = ns;
+        if (tid == kQReq - 1) {
+            uint32_t ns = 0;
+            unsigned long long tot = 0;
+            for (int q = 0; q < kQReq; ++q)
+                if (req_first[q] == q) { ++ns; tot += req_cnt[q]; }
+            ctrl->slot_off[ns] = tot;
+            ctrl->nslots = ns;
+        }
     }
 }
 
-// one block per slot: radix select (4 passes of 8 bits) of every request that lives in this slot
-__global__ void __launch_bounds__(256)
+// one block per slot: radix select (4 passes of 8 bits) of every request that lives in this slot.
+// The keys of a slot lie in one narrow bin, so most of them share their leading digits: equal
+// digits within a warp are counted once (match), which keeps the shared-memory atomics apart.
+__global__ void __launch_bounds__(1024)
 quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sh_prefix, sh_mask;
     __shared__ unsigned long long sh_k;
+    __shared__ uint32_t req_slot[kQReq];
+    __shared__ unsigned long long req_local[kQReq];
     const uint32_t slot = blockIdx.x;
     if (slot >= ctrl->nslots) return;
+    if (threadIdx.x < kQReq) {
+        req_slot[threadIdx.x] = ctrl->req_slot[threadIdx.x];
+        req_local[threadIdx.x] = ctrl->req_local[threadIdx.x];
+    }
     const uint32_t* keys = list + ctrl->slot_off[slot];
     const unsigned long long n = ctrl->slot_off[slot + 1] - ctrl->slot_off[slot];
+    const unsigned long long n_up = (n + blockDim.x - 1) / blockDim.x * blockDim.x;
+    const int lane = threadIdx.x & 31;
+    __syncthreads();
     for (int q = 0; q < kQReq; ++q) {
-        if (ctrl->req_slot[q] != slot) continue;           // uniform across the block
-        if (threadIdx.x == 0) { sh_prefix = 0; sh_mask = 0; sh_k = ctrl->req_local[q]; }
+        if (req_slot[q] != slot) continue;                 // uniform across the block
+        if (threadIdx.x == 0) { sh_prefix = 0; sh_mask = 0; sh_k = req_local[q]; }
         __syncthreads();
         for (int shift = 24; shift >= 0; shift -= 8) {
-            hist[threadIdx.x] = 0;
+            if (threadIdx.x < 256) hist[threadIdx.x] = 0;
             __syncthreads();
             const uint32_t prefix = sh_prefix, mask = sh_mask;
-            for (unsigned long long i = threadIdx.x; i < n; i += blockDim.x) {
-                const uint32_t k = keys[i];
-                if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFFu], 1u);
+            for (unsigned long long i0 = threadIdx.x; i0 < n_up; i0 += 4ull * blockDim.x) {
+                uint32_t kk[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {               // four independent loads in flight
+                    const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
+                    kk[u] = i < n ? keys[i] : 0u;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
+                    if (i >= n_up) break;                  // uniform over the block
+                    const uint32_t k = kk[u];
+                    const bool sel = i < n && (k & mask) == prefix;
+                    const unsigned act = __ballot_sync(0xFFFFFFFFu, sel);
+                    if (sel) {
+                        const uint32_t d = (k >> shift) & 0xFFu;
+                        const unsigned peers = __match_any_sync(act, d);
+                        if (lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+                    }
+                }
             }
             __syncthreads();
             if (threadIdx.x == 0) {
@@ -249,22 +388,22 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     cudaError_t e;
     set_requests_kernel<<<1, 64, 0, st>>>(ws.ctrl, rq);
     if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) return e;
-    const int blocks = sm_count() * 2;
+    const int blocks = sm_count() * 3;
     const size_t sm0 = kQBins * sizeof(uint32_t);
     if (mode == AAAC_INT4) {
-        if ((e = cudaFuncSetAttribute(quantile_scan_kernel<AAAC_INT4, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
-        quantile_scan_kernel<AAAC_INT4, 0><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist, nullptr, nullptr);
+        if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_INT4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
+        quantile_hist_kernel<AAAC_INT4><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
     } else {
-        if ((e = cudaFuncSetAttribute(quantile_scan_kernel<AAAC_NVFP4, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
-        quantile_scan_kernel<AAAC_NVFP4, 0><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist, nullptr, nullptr);
+        if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_NVFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
+        quantile_hist_kernel<AAAC_NVFP4><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
     }
     quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qprefix, ws.qslot_of_bin);
-    const int blocks1 = sm_count() * 8;
+    const int blocks1 = sm_count() * 4;
     if (mode == AAAC_INT4)
-        quantile_scan_kernel<AAAC_INT4, 1><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, nullptr, ws.qslot_of_bin, ws.qlist);
+        quantile_collect_kernel<AAAC_INT4><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qslot_of_bin, ws.qlist);
     else
-        quantile_scan_kernel<AAAC_NVFP4, 1><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, nullptr, ws.qslot_of_bin, ws.qlist);
-    quantile_select_kernel<<<kQReq, 256, 0, st>>>(ws.ctrl, ws.qlist);
+        quantile_collect_kernel<AAAC_NVFP4><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qslot_of_bin, ws.qlist);
+    quantile_select_kernel<<<kQReq, 1024, 0, st>>>(ws.ctrl, ws.qlist);
     quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl);
     return cudaGetLastError();
 }
