@@ -30,7 +30,10 @@
 //     |E_r - E_r,exact| <= 2^-24 * 16 E_r + 2 eta sum I |u_r| and
 //     sum I |u_r| <= sqrt(sum I * E_r).  Groups with
 //     |E0 - E1| <= 2^-24 (16 (E0 + E1) + 2.83 * 32 max|T| sqrt(sum I (E0 + E1))) (and NaN) are
-//     re-evaluated in double with the exact entries, so sigma is the double-precision decision.
+//     re-evaluated in double with the exact entries, so sigma is the double-precision decision
+//     (the kernel tests against the slightly larger bound that sqrt(a b) <= a / 16 + 4 b gives,
+//     which needs one multiply-add per group).  The two errors are carried as one packed
+//     FP32 pair per weight (sub / mul / fma.f32x2).
 // (c) Centroid sums, centred.  Lane-private shared-memory bins [sigma][entry] hold
 //     (sum I (x - c), sum I) with c the constant of (b) for the entry the weight is assigned to,
 //     so the new entry is c + sum I (x - c) / sum I.  The residual sums are small and of mixed
@@ -68,6 +71,17 @@ struct FitParams {
     int n_rounds;
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
 };
+
+// hi + lo += v, error-free (Knuth's two-sum in FP32; the intrinsics keep the compiler from
+// re-associating).  Double-precision arithmetic is slow on this GPU, so the in-kernel
+// reductions carry their sums as FP32 pairs and convert once at the end.
+__device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
+    const float s = __fadd_rn(hi, v);
+    const float bb = __fsub_rn(s, hi);
+    const float err = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(v, bb));
+    hi = s;
+    lo = __fadd_rn(lo, err);
+}
 
 constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
 
@@ -164,15 +178,17 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
   for (int round = 0; round < p.n_rounds; ++round) {
     build_tables<MODE, NW, REP>(S, dyn);
     for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
-    const float tmax283 = S.tmax283;
+    // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
+    // most g1 * (E0 + E1) + g2 * sum I, with kappa = 1/8 (about the usual |w~ - entry|)
+    const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
     double Eacc = 0.0;
 
     int cur_slab = -1;
-    float Iv[8];
-    float isum = 0.f;         // sum of I over the lane's group (rounded up a little)
+    uint64_t II[8];           // {I, I} of the lane's eight columns
+    float isum = 0.f;         // g2 * sum of I over the lane's group (rounded up a little)
     bool col_ok = false;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
+    for (int j = 0; j < 8; ++j) II[j] = 0ull;
 
     // (slab, row block) of the current item and of the one being loaded
     int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
@@ -193,20 +209,20 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             const int col0 = slab * 256 + lane * 8;
             col_ok = col0 < K;
             isum = 0.f;
+            float Iv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
             if (col_ok) {
                 const float4 a = __ldg(reinterpret_cast<const float4*>(p.I + col0));
                 const float4 b = __ldg(reinterpret_cast<const float4*>(p.I + col0 + 4));
                 Iv[0] = a.x; Iv[1] = a.y; Iv[2] = a.z; Iv[3] = a.w;
                 Iv[4] = b.x; Iv[5] = b.y; Iv[6] = b.z; Iv[7] = b.w;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) isum += Iv[j];
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
             }
 #pragma unroll
+            for (int j = 0; j < 8; ++j) { isum += Iv[j]; II[j] = pack2(Iv[j], Iv[j]); }
+#pragma unroll
             for (int o = LPG / 2; o; o >>= 1) isum += __shfl_xor_sync(0xFFFFFFFFu, isum, o);
-            isum *= 1.0001f;
+            isum = __fmul_ru(isum * 1.0001f, g2);
         }
         const int row0 = rb * kRowsPerItem + warp * R;
         const int nrows = min(R, N - row0);                // rows of this warp inside the layer (may be <= 0)
@@ -216,9 +232,10 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         // bins of one row runs while the table lookups of the next row are in flight:
         //   L1(u): w~ and the loads of {J_low, thr};   L2(u): slot and the loads of {P, Q};
         //   M(u):  errors, sigma, the centred terms and bin addresses;   B(u): bins += terms.
+        float eitem = 0.f;                                 // objective of this item's groups led by this lane
         float x[8];                                        // w~ of the row in L1..M
         uint2 e1v[8];                                      // {J_low * 256, thr}
-        float2 pq[8];                                      // {P, Q}
+        uint64_t pq[8];                                    // {P, Q}, packed
         float mt[8];                                       // chosen centred term I (x - c) of the row in B
         uint32_t ba[8];                                    // its bin address
         auto L1 = [&](int u) {
@@ -234,56 +251,54 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         auto L2 = [&]() {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                pq[j] = lds_table_f2(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
+                pq[j] = lds_table_b64(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
         };
         auto M = [&](int u) {
-            float m0[8], m1[8];
-            float e0 = 0.f, e1 = 0.f;
+            uint64_t m[8];                                 // {I (x - P), I (x - Q)}
+            uint64_t e01 = 0ull;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float u0 = __fsub_rn(x[j], pq[j].x), u1 = __fsub_rn(x[j], pq[j].y);
-                m0[j] = __fmul_rn(Iv[j], u0);
-                m1[j] = __fmul_rn(Iv[j], u1);
-                e0 = __fmaf_rn(m0[j], u0, e0);
-                e1 = __fmaf_rn(m1[j], u1, e1);
+                const uint64_t u01 = sub2(pack2(x[j], x[j]), pq[j]);
+                m[j] = mul2(II[j], u01);
+                e01 = fma2(m[j], u01, e01);
             }
+            float e0 = lo2(e01), e1 = hi2(e01);
 #pragma unroll
             for (int s = LPG / 2; s; s >>= 1) {
                 e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, s);
                 e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, s);
             }
             const float es = e0 + e1;
-            const float tau = 0x1p-24f * __fmaf_rn(tmax283, __fsqrt_ru(__fmul_ru(isum, es)), 16.f * es);
+            const float tau = __fmaf_ru(es, g1, isum);
             // lanes past K carry I = 0 and w~ = 0; they need the exact path only if their slot is
             // poisoned (NaN), so that no NaN reaches a bin
             const bool near = !(fabsf(e1 - e0) > tau) && (col_ok || !(es == es));
             bool sg = e1 < e0;
-            double emin = (double)(sg ? e1 : e0);
+            float emin = sg ? e1 : e0;
             if (__any_sync(0xFFFFFFFFu, near)) {
                 // near-ties and poisoned slots: decide in double (rare, out of line), then redo
                 // this lane's centred terms from the intervals that call has found
                 Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = Iv[j]; }
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); }
                 const Exact8 ex = exact_groups<LPG>(&S, r, (int)near);
                 if (near) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        pq[j] = lds_table_f2((uint32_t)(c0 + ex.J[j] * kSlotBytes));
-                        m0[j] = __fmul_rn(Iv[j], __fsub_rn(x[j], pq[j].x));
-                        m1[j] = __fmul_rn(Iv[j], __fsub_rn(x[j], pq[j].y));
+                        pq[j] = lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes));
+                        m[j] = mul2(II[j], sub2(pack2(x[j], x[j]), pq[j]));
                     }
                     sg = ex.sigma != 0;
-                    emin = ex.emin;
+                    emin = (float)ex.emin;
                 }
             }
-            if (col_ok && (lane % LPG) == 0) Eacc += emin;
+            if (col_ok && (lane % LPG) == 0) eitem += emin;
             // cell = entry index (low bits of the centre constant) under the chosen table
             const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                mt[j] = sg ? m1[j] : m0[j];
-                ba[j] = base + (__float_as_uint(sg ? pq[j].y : pq[j].x) & kIdxMask) * kSlotBytes;
+                mt[j] = sg ? hi2(m[j]) : lo2(m[j]);
+                ba[j] = base + ((sg ? (uint32_t)(pq[j] >> 32) : (uint32_t)pq[j]) & kIdxMask) * kSlotBytes;
             }
         };
         auto B = [&](int j0, int j1) {
@@ -291,7 +306,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             for (int j = j0; j < j1; ++j) {
                 float2 a = lds_bin(ba[j]);
                 a.x += mt[j];
-                a.y += Iv[j];
+                a.y += lo2(II[j]);
                 sts_bin(ba[j], a);
             }
         };
@@ -312,7 +327,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                     for (int j = j0; j < j1; ++j) {
                         float2 a = lds_bin(ba_prev[j]);
                         a.x += mt_prev[j];
-                        a.y += Iv[j];
+                        a.y += lo2(II[j]);
                         sts_bin(ba_prev[j], a);
                     }
                 };
@@ -340,32 +355,35 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 B(0, 8);
             }
         }
+        Eacc += (double)eitem;
     }
 
     // ---- block partial: lane c of a warp adds the 32 lane-private values of cell c (in a
     //      rotated, fixed order that avoids bank conflicts); then the warps are added ----
     __syncthreads();                                       // every warp is done with the lookup tables
     {
-        double sx = 0.0, sy = 0.0;
+        float hx = 0.f, lx = 0.f, hy = 0.f, ly = 0.f;
 #pragma unroll 4
         for (int i = 0; i < 32; ++i) {
             const float2 a = lds_bin(bins_warp + lane * kSlotBytes + ((i + lane) & 31) * 8);
-            sx += (double)a.x;
-            sy += (double)a.y;
+            two_sum(hx, lx, a.x);
+            two_sum(hy, ly, a.y);
         }
-        wsum[warp * kPartStride + lane] = sx;
-        wsum[warp * kPartStride + kCells + lane] = sy;
+        wsum[warp * kPartStride + lane] = (double)hx + (double)lx;
+        wsum[warp * kPartStride + kCells + lane] = (double)hy + (double)ly;
     }
 #pragma unroll
     for (int s = 16; s; s >>= 1) Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, s);
     if (lane == 0) wsum[warp * kPartStride + 2 * kCells] = Eacc;
     __syncthreads();
-    double* part = p.part + (size_t)(round & 1) * kMaxBlocks * kPartStride;
+    // a partial is stored as an FP32 pair (hi, lo) of its double value: exact to 2^-48
+    float2* part = reinterpret_cast<float2*>(p.part + (size_t)(round & 1) * kMaxBlocks * kPartStride);
     if (tid < kUsed) {
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < NW; ++w) s += wsum[w * kPartStride + tid];
-        part[(size_t)blockIdx.x * kPartStride + tid] = s;
+        const float hi = (float)s;
+        part[(size_t)blockIdx.x * kPartStride + tid] = make_float2(hi, (float)(s - (double)hi));
     }
 
     // ---- all blocks meet; then each adds the partials of all blocks in the same fixed order
@@ -378,10 +396,14 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         constexpr int kStrands = NT / kUsed;
         const int strand = tid / kUsed, val = tid - strand * kUsed;
         if (strand < kStrands) {
-            double s = 0.0;
-#pragma unroll 8
-            for (unsigned b = strand; b < gridDim.x; b += kStrands) s += __ldcg(part + (size_t)b * kPartStride + val);
-            wsum[strand * kPartStride + val] = s;
+            float hi = 0.f, lo = 0.f;
+#pragma unroll 4
+            for (unsigned b = strand; b < gridDim.x; b += kStrands) {
+                const float2 v = __ldcg(part + (size_t)b * kPartStride + val);
+                two_sum(hi, lo, v.x);
+                lo = __fadd_rn(lo, v.y);
+            }
+            wsum[strand * kPartStride + val] = (double)hi + (double)lo;
         }
         __syncthreads();
         if (tid < kUsed) {
@@ -392,22 +414,21 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         }
     }
     __syncthreads();
-    double tnew = 0.0;
-    int rank = 0;
     if (tid < 2 * kM) {
         // cells of duplicate entries are empty: they keep their value
         const double sx = S.tot[tid], wt = S.tot[kCells + tid];
-        tnew = (wt > 0.0) ? (double)S.centre[tid] + __ddiv_rn(sx, wt) : S.Td[tid];
-        // ascending order within the table by rank (ties by index)
-        const int r = tid & 16;
-        for (int i = 0; i < kM; ++i) {
-            const double sxi = S.tot[r + i], wti = S.tot[kCells + r + i];
-            const double ti = (wti > 0.0) ? (double)S.centre[r + i] + __ddiv_rn(sxi, wti) : S.Td[r + i];
-            rank += (ti < tnew) || (ti == tnew && i < (tid & 15));
-        }
+        S.tot[2 * kCells + 1 + tid] = (wt > 0.0) ? (double)S.centre[tid] + __ddiv_rn(sx, wt) : S.Td[tid];
     }
     __syncthreads();
-    if (tid < 2 * kM) S.Td[(tid & 16) + rank] = tnew;
+    if (tid < 2 * kM) {
+        // ascending order within the table by rank (ties by index)
+        const double* tn = S.tot + 2 * kCells + 1 + (tid & 16);
+        const double t = tn[tid & 15];
+        int rank = 0;
+#pragma unroll 1
+        for (int i = 0; i < kM; ++i) rank += (tn[i] < t) || (tn[i] == t && i < (tid & 15));
+        S.Td[(tid & 16) + rank] = t;
+    }
     if (blockIdx.x == 0 && tid == 0 && p.err_trace) p.err_trace[round] = S.tot[2 * kCells];
     __syncthreads();
   }
