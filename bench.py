@@ -47,13 +47,15 @@ def peaks():
 
 
 def measured_traffic_per_weight():
-    """DRAM bytes per weight of the fit-round kernel from the committed ncu summary, if any."""
-    p = os.path.join(ROOT, "profiles", "fit_round_traffic.json")
-    if os.path.exists(p):
-        try:
-            return float(json.load(open(p))["dram_bytes_per_weight"])
-        except Exception:
-            return None
+    """DRAM bytes per weight and round of the fit-rounds kernel, from the line
+    `dram_bytes_per_weight_round = X` of the committed ncu summary (None if absent)."""
+    p = os.path.join(ROOT, "profiles", "fit_rounds_cfg2_gate_proj.md")
+    try:
+        for line in open(p):
+            if line.strip().startswith("dram_bytes_per_weight_round"):
+                return float(line.split("=")[1].split()[0])
+    except Exception:
+        pass
     return None
 
 
@@ -109,21 +111,25 @@ def make_layers(seed, names=None):
     return [synth.config2_layer(w, seed=seed, tokens=TOKENS) for w in (names or LAYERS)]
 
 
-def cpu_baseline_sample(layers, rounds=ROUNDS, rows=4096):
-    """The oracle, as it stands, on a bounded sample: the first `rows` rows of q_proj, scales +
-    quantile init excluded, `rounds` fit rounds timed on all host cores (about 15 core-seconds)."""
+def cpu_baseline_sample(layers, rounds=ROUNDS, rows=None):
+    """The oracle, as it stands, on a bounded sample of the workload: the fit rounds (scales and
+    quantile init excluded) of the given layers, optionally only their first `rows` rows, on all
+    host cores."""
     import oracle
-    c = layers[0]
-    W = np.ascontiguousarray(c["W"][:rows])
-    I = oracle.act_stats(c["X"][:256])
-    s, ts = oracle.scales(W, c["mode"], c["group"])
-    wt = oracle.normalise(W, c["mode"], c["group"], s, ts)
-    T = oracle.init_quantile(wt)
-    t0 = time.perf_counter()
-    for _ in range(rounds):
-        T, _ = oracle.fit_round(wt, I, c["group"], T)
-    dt = time.perf_counter() - t0
-    return W.size * rounds / dt / 1e9, oracle.max_threads(), f"q_proj rows 0..{rows - 1} x 4096, {rounds} fit rounds", dt
+    total_w, dt, names = 0, 0.0, []
+    for c in layers:
+        W = np.ascontiguousarray(c["W"][:rows]) if rows else c["W"]
+        I = oracle.act_stats(c["X"][:256])
+        s, ts = oracle.scales(W, c["mode"], c["group"])
+        wt = oracle.normalise(W, c["mode"], c["group"], s, ts)
+        T = oracle.init_quantile(wt)
+        t0 = time.perf_counter()
+        for _ in range(rounds):
+            T, _ = oracle.fit_round(wt, I, c["group"], T)
+        dt += time.perf_counter() - t0
+        total_w += W.size
+        names.append(f"{c['name'].split('/')[-1]} {W.shape[0]}x{W.shape[1]}")
+    return total_w * rounds / dt / 1e9, oracle.max_threads(), f"{rounds} fit rounds of " + ", ".join(names), dt
 
 
 def run_reference(args, rank):

@@ -310,16 +310,34 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
                 }
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                unsigned long long k = sh_k;
-                int d = 0;
-                for (; d < 255; ++d) {
-                    if (k < hist[d]) break;
-                    k -= hist[d];
+            if (threadIdx.x < 32) {
+                // digit that holds rank k: lane l owns digits 8 l .. 8 l + 7
+                uint32_t c[8], tot = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { c[i] = hist[lane * 8 + i]; tot += c[i]; }
+                uint32_t incl = tot;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += t;
                 }
-                sh_k = k;
-                sh_prefix = prefix | ((uint32_t)d << shift);
-                sh_mask = mask | (0xFFu << shift);
+                const unsigned long long k = sh_k;
+                const unsigned long long before = incl - tot;
+                const bool mine = k >= before && k < (unsigned long long)incl;
+                const unsigned who = __ballot_sync(0xFFFFFFFFu, mine);
+                // ranks beyond the list (never requested) fall to the last digit
+                const int owner = who ? __ffs(who) - 1 : 31;
+                if (lane == owner) {
+                    unsigned long long r = k - before;
+                    int i = 0;
+                    for (; i < 7; ++i) {
+                        if (r < c[i]) break;
+                        r -= c[i];
+                    }
+                    sh_k = r;
+                    sh_prefix = prefix | ((uint32_t)(lane * 8 + i) << shift);
+                    sh_mask = mask | (0xFFu << shift);
+                }
             }
             __syncthreads();
         }
