@@ -174,7 +174,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2605_08692_b200 import binding, build
+    from paper_2605_08692_b200 import binding, build, sharding
     build.build()
     binding.lib()
     if not torch.cuda.is_available():
@@ -186,7 +186,7 @@ def main():
 
     warmup = max(args.warmup, 3)
     names = [n for n in args.layers.split(",") if n]
-    layers = make_layers(seed=rank, names=names)
+    layers = make_layers(seed=sharding.seed_for_rank(0, rank), names=names)
     mode = layers[0]["mode"]
 
     def to_dev(a):
@@ -242,12 +242,9 @@ def main():
     clocks = sampler.stop() if sampler else None
     if int(status.item()) != 0:
         raise SystemExit("device status reports non-finite input")
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
-    value = world * weights_per_step * ROUNDS / (ms_step * 1e-3) / 1e9
+    value = sharding.job_throughput(weights_per_step, ROUNDS, ms_step, world)
 
     # roofline of the dominant kernel: algorithmic bytes of every timed fit-round launch / its device time
     per_launch_w = []
@@ -293,13 +290,10 @@ def main():
             host_step()
         e1.record()
         barrier()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item()) / args.steps
+        ms_e2e = sharding.max_over_ranks(e0.elapsed_time(e1), dev) / args.steps
         h2d = sum(h["W"].numel() * 2 + h["X"].numel() * 2 for h in host)
         d2h = sum(h["codes"].numel() + h["sc"].numel() + 128 + 64 + 4 + 16 + 4 for h in host)
-        e2e = {"value": world * weights_per_step * ROUNDS / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+        e2e = {"value": sharding.job_throughput(weights_per_step, ROUNDS, ms_e2e, world), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ms_e2e}
     except Exception as ex:                                   # report, never hide
         e2e = {"value": None, "unit": UNIT, "error": repr(ex)}

@@ -2,9 +2,11 @@
 //
 // Layout: X is [T x K] BF16 row-major.  A block covers 256 adjacent columns (each lane owns
 // 8 of them = one 128-bit load per row) and a strip of rows; its 8 warps take rows
-// round-robin.  The square of a BF16 value is exact in double, and every partial sum is
-// kept in double, so the result differs from an index-order double sum only by double
-// rounding; a second kernel adds the strip partials in strip order and rounds once to FP32.
+// round-robin.  The square of a BF16 value is exact in FP32 (16 significant bits); a thread adds
+// its squares error-free into an FP32 pair (two-sum), because double-precision arithmetic runs
+// at a small fraction of the FP32 rate on this GPU.  The pairs become doubles once per thread,
+// so the result differs from an index-order double sum only by rounding at the 2^-48 level; a
+// second kernel adds the strip partials in strip order and rounds once to FP32.
 #include <mutex>
 
 #include "internal.cuh"
@@ -16,6 +18,24 @@ namespace {
 constexpr int kWarps = 8;
 constexpr int kUnroll = 4;
 
+// hi + lo += v without rounding error (Knuth's two-sum; intrinsics so that nothing is re-associated)
+__device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
+    const float s = __fadd_rn(hi, v);
+    const float bb = __fsub_rn(s, hi);
+    const float err = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(v, bb));
+    hi = s;
+    lo = __fadd_rn(lo, err);
+}
+__device__ __forceinline__ void add_squares(float (&hi)[8], float (&lo)[8], uint4 v) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float a = bf16_lo(w[j]), b = bf16_hi(w[j]);
+        two_sum(hi[2 * j], lo[2 * j], __fmul_rn(a, a));
+        two_sum(hi[2 * j + 1], lo[2 * j + 1], __fmul_rn(b, b));
+    }
+}
+
 __global__ void __launch_bounds__(kWarps * 32)
 act_sumsq_kernel(const uint16_t* __restrict__ X, int64_t T, int64_t K, int64_t ldx,
                  double* __restrict__ part, int rows_per_split) {
@@ -25,9 +45,9 @@ act_sumsq_kernel(const uint16_t* __restrict__ X, int64_t T, int64_t K, int64_t l
     const bool active = col0 < K;
     const int64_t t_begin = (int64_t)blockIdx.y * rows_per_split;
     const int64_t t_end = min(T, t_begin + rows_per_split);
-    double acc[8];
+    float hi[8], lo[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.0;
+    for (int j = 0; j < 8; ++j) { hi[j] = 0.f; lo[j] = 0.f; }
 
     if (active) {
         const uint16_t* base = X + col0;
@@ -38,29 +58,12 @@ act_sumsq_kernel(const uint16_t* __restrict__ X, int64_t T, int64_t K, int64_t l
             for (int u = 0; u < kUnroll; ++u)
                 v[u] = __ldcs(reinterpret_cast<const uint4*>(base + (t + u * kWarps) * ldx));
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    double a = (double)bf16_lo(w[j]), b = (double)bf16_hi(w[j]);
-                    acc[2 * j] = fma(a, a, acc[2 * j]);
-                    acc[2 * j + 1] = fma(b, b, acc[2 * j + 1]);
-                }
-            }
+            for (int u = 0; u < kUnroll; ++u) add_squares(hi, lo, v[u]);
         }
-        for (; t < t_end; t += kWarps) {
-            uint4 v = __ldcs(reinterpret_cast<const uint4*>(base + t * ldx));
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                double a = (double)bf16_lo(w[j]), b = (double)bf16_hi(w[j]);
-                acc[2 * j] = fma(a, a, acc[2 * j]);
-                acc[2 * j + 1] = fma(b, b, acc[2 * j + 1]);
-            }
-        }
+        for (; t < t_end; t += kWarps) add_squares(hi, lo, __ldcs(reinterpret_cast<const uint4*>(base + t * ldx)));
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = acc[j];
+    for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = (double)hi[j] + (double)lo[j];
     __syncthreads();
     const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (col < K) {
