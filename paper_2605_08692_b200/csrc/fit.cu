@@ -297,8 +297,11 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                mt[j] = sg ? hi2(m[j]) : lo2(m[j]);
-                ba[j] = base + ((sg ? (uint32_t)(pq[j] >> 32) : (uint32_t)pq[j]) & kIdxMask) * kSlotBytes;
+                float m0, m1, cP, cQ;
+                unpack2(m[j], m0, m1);
+                unpack2(pq[j], cP, cQ);
+                mt[j] = sg ? m1 : m0;
+                ba[j] = base + (__float_as_uint(sg ? cQ : cP) & kIdxMask) * kSlotBytes;
             }
         };
         auto B = [&](int j0, int j1) {
