@@ -43,6 +43,19 @@ struct PackParams {
     int items, per_block, nrb;
 };
 
+// Number of the row's weights that lie exactly half-way between two different entries of the
+// chosen table (rare; kept out of line so that the hot loop stays small).
+__device__ __noinline__ int count_idx_ties(const FitTables* S, Row8 r, int sg) {
+    int n = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll 1
+        for (int jj = 0; jj < kNBP; ++jj)
+            if (S->bp[jj] == r.x[j] && S->src[jj] == (uint8_t)sg && S->exact[jj]) { ++n; break; }
+    }
+    return n;
+}
+
 template <int MODE, int NW, int REP>
 __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
@@ -230,11 +243,10 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
             }
             Eout += (double)eo;
             if (tcand) {
-                // weights exactly half-way between two different entries of the chosen table
+                Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    for (int jj = 0; jj < kNBP; ++jj)
-                        if (S.bp[jj] == x[j] && S.src[jj] == (uint8_t)sg && S.exact[jj]) { ++n_idx_tie; break; }
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = 0.f; }
+                n_idx_tie += count_idx_ties(&S, r, (int)sg);
             }
             *reinterpret_cast<uint32_t*>(p.codes + (((size_t)row * (size_t)K + col0) >> 1)) = word;
             if ((lane % LPG) == 0) {
