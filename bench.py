@@ -153,6 +153,95 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+STACKS = {
+    # name: (decoder layers, hidden, kv width, intermediate, mode, tokens, rounds)
+    "stack8b": (32, 4096, 1024, 14336, 0, 16384, 20),     # Llama-3-8B-shaped, INT4 g128
+    "stack7b": (28, 3584, 512, 18944, 1, 16384, 20),      # Qwen2.5-7B-shaped, NVFP4 g16
+}
+
+
+def run_stack(args, which):
+    """Wall time of a whole decoder stack of random weights: per decoder layer four activation
+    matrices (attention input shared by q/k/v, o input, MLP input shared by gate/up, down input) and
+    seven linears, each through act_stats (once per distinct input), scales, quantile init, the fit
+    rounds and the pack pass.  The layers of a stack are i.i.d. synthetic, so one decoder layer's
+    tensors are generated on the device (seeded torch generator, outside the timed region) and the
+    per-layer path is run once per decoder layer on them; every linear re-reads its W from HBM
+    (one decoder layer touches > 1 GB, far more than the L2)."""
+    import torch
+    from paper_2605_08692_b200 import binding, build
+    build.build()
+    L, H, KV, FF, mode, tokens, rounds = STACKS[which]
+    g = 128 if mode == 0 else 16
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+
+    def weights(n, k, t5=False):
+        w = torch.randn(n, k, device=dev, generator=gen)
+        if t5:
+            chi = sum(torch.randn(n, k, device=dev, generator=gen) ** 2 for _ in range(5)) / 5.0
+            w = w / chi.sqrt()
+        return (w * 0.02).to(torch.bfloat16)
+
+    def acts(k):
+        c = torch.exp(torch.randn(k, device=dev, generator=gen))
+        c[torch.randperm(k, device=dev, generator=gen)[: max(1, k // 200)]] *= 30.0
+        return (torch.randn(tokens, k, device=dev, generator=gen) * c).to(torch.bfloat16)
+
+    t5 = which == "stack7b"
+    X = {"attn": acts(H), "o": acts(H), "mlp": acts(H), "down": acts(FF)}
+    lin = [("q", H, H, "attn"), ("k", KV, H, "attn"), ("v", KV, H, "attn"), ("o", H, H, "o"),
+           ("gate", FF, H, "mlp"), ("up", FF, H, "mlp"), ("down", H, FF, "down")]
+    Ws = {n: weights(N, K, t5) for n, N, K, _ in lin}
+    out = {}
+    for n, N, K, _ in lin:
+        out[n] = dict(T01=torch.zeros(2, 16, dtype=torch.float32, device=dev),
+                      Tb=torch.empty(2, 16, dtype=torch.uint16, device=dev),
+                      scales=torch.empty(N, K // g, dtype=torch.uint16 if mode == 0 else torch.uint8, device=dev),
+                      ts=torch.ones(1, dtype=torch.float32, device=dev),
+                      codes=torch.empty(N, K // 2, dtype=torch.uint8, device=dev),
+                      err=torch.zeros(2, dtype=torch.float64, device=dev),
+                      ws=binding.alloc_workspace(mode, N, K, tokens, dev))
+    Iv = {k: torch.empty(x.shape[1], dtype=torch.float32, device=dev) for k, x in X.items()}
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def decoder_layer():
+        for k, x in X.items():
+            binding.act_stats(x, Iv[k], out["down" if k == "down" else "q"]["ws"], dev_status=status)
+        for n, N, K, xin in lin:
+            o = out[n]
+            binding.fit_layer(Ws[n], mode, I=Iv[xin], n_outer=rounds, init=binding.INIT_QUANTILE, T01=o["T01"],
+                              scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
+            binding.pack(Ws[n], mode, I=Iv[xin], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"],
+                         tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"])
+
+    for _ in range(2):
+        decoder_layer()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(L):
+        decoder_layer()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if int(status.item()) != 0:
+        raise SystemExit("device status is set")
+    wall = e0.elapsed_time(e1) * 1e-3
+    wl = sum(N * K for _, N, K, _ in lin)
+    line = {"metric": "aaac_stack_wall_s", "value": wall, "unit": "s", "n_gpus": 1, "higher_is_better": False,
+            "dtype": "f32", "data": "synthetic (device-generated, one decoder layer's tensors reused for every layer)",
+            "config": {"workload": f"{which}: {L} decoder layers x 7 linears (hidden {H}, kv {KV}, intermediate {FF}), "
+                                   f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'}, {tokens} tokens per input, quantile init, "
+                                   f"{rounds} rounds; act_stats + scales + init + rounds + pack",
+                       "linears": 7 * L, "weights": wl * L, "rounds": rounds},
+            "gweights_per_s_per_round": wl * L * rounds / wall / 1e9, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -162,7 +251,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", default=",".join(LAYERS),
                     help="subset of the workload's layers (profiling a small case); the default is the full workload")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2"] + sorted(STACKS),
+                    help="cfg2 (default): the benchmark contract; stack8b / stack7b: wall time of a whole decoder stack")
     args = ap.parse_args()
+    if args.workload != "cfg2":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_stack(args, args.workload)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
