@@ -236,8 +236,8 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         float x[8];                                        // w~ of the row in L1..M
         uint2 e1v[8];                                      // {J_low * 256, thr}
         uint64_t pq[8];                                    // {P, Q}, packed
-        float mt[8];                                       // chosen centred term I (x - c) of the row in B
-        uint32_t ba[8];                                    // its bin address
+        float mt[2][8];                                    // chosen centred term I (x - c) of the rows in B / M
+        uint32_t ba[2][8];                                 // its bin address
         auto L1 = [&](int u) {
             const float rinv = MODE == AAAC_NVFP4 ? S.rlut[sc[u] & 0x7Fu] : __uint_as_float(sc[u]);
             const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             for (int j = 0; j < 8; ++j)
                 pq[j] = lds_table_b64(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
         };
-        auto M = [&](int u) {
+        auto M = [&](int u, float (&mt_o)[8], uint32_t (&ba_o)[8]) {
             uint64_t m[8];                                 // {I (x - P), I (x - Q)}
             uint64_t e01 = 0ull;
 #pragma unroll
@@ -300,17 +300,17 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 float m0, m1, cP, cQ;
                 unpack2(m[j], m0, m1);
                 unpack2(pq[j], cP, cQ);
-                mt[j] = sg ? m1 : m0;
-                ba[j] = base + (__float_as_uint(sg ? cQ : cP) & kIdxMask) * kSlotBytes;
+                mt_o[j] = sg ? m1 : m0;
+                ba_o[j] = base + (__float_as_uint(sg ? cQ : cP) & kIdxMask) * kSlotBytes;
             }
         };
-        auto B = [&](int j0, int j1) {
+        auto B = [&](const float (&mt_i)[8], const uint32_t (&ba_i)[8], int j0, int j1) {
 #pragma unroll
             for (int j = j0; j < j1; ++j) {
-                float2 a = lds_bin(ba[j]);
-                a.x += mt[j];
+                float2 a = lds_bin(ba_i[j]);
+                a.x += mt_i[j];
                 a.y += lo2(II[j]);
-                sts_bin(ba[j], a);
+                sts_bin(ba_i[j], a);
             }
         };
 
@@ -318,29 +318,17 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
             L1(0);
             L2();
-            M(0);
+            M(0, mt[0], ba[0]);
 #pragma unroll
             for (int u = 1; u < R; ++u) {
-                float mt_prev[8];
-                uint32_t ba_prev[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { mt_prev[j] = mt[j]; ba_prev[j] = ba[j]; }
-                auto Bprev = [&](int j0, int j1) {
-#pragma unroll
-                    for (int j = j0; j < j1; ++j) {
-                        float2 a = lds_bin(ba_prev[j]);
-                        a.x += mt_prev[j];
-                        a.y += lo2(II[j]);
-                        sts_bin(ba_prev[j], a);
-                    }
-                };
+                const int prev = (u - 1) & 1, cur = u & 1;
                 L1(u);
-                Bprev(0, 4);
+                B(mt[prev], ba[prev], 0, 4);
                 L2();
-                Bprev(4, 8);
-                M(u);
+                B(mt[prev], ba[prev], 4, 8);
+                M(u, mt[cur], ba[cur]);
             }
-            B(0, 8);
+            B(mt[(R - 1) & 1], ba[(R - 1) & 1], 0, 8);
         } else {
             // ragged last row block of the layer: row by row
             for (int u = 0; u < nrows; ++u) {
@@ -354,8 +342,8 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 sc[0] = ss;
                 L1(0);
                 L2();
-                M(0);
-                B(0, 8);
+                M(0, mt[0], ba[0]);
+                B(mt[0], ba[0], 0, 8);
             }
         }
         Eacc += (double)eitem;

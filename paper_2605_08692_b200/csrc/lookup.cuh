@@ -173,7 +173,7 @@ struct Exact8 { int J[8]; double emin; int sigma; int tie; };
 
 // Double-precision decision (Eq. 8 as a plain double-precision loop states it, lanes of a group
 // combined by a shuffle tree) for the groups whose lanes pass need != 0; every lane of the warp
-// calls.  The interval of every weight is found by direct search of the breakpoint list.
+// calls.  The interval of every weight is found by binary search of the breakpoint list.
 template <int LPG>
 __device__ __noinline__ Exact8 exact_groups(const FitTables* S, Row8 r, int need) {
     Exact8 out;
@@ -182,8 +182,9 @@ __device__ __noinline__ Exact8 exact_groups(const FitTables* S, Row8 r, int need
     for (int j = 0; j < 8; ++j) {
         int J = 0;
         if (need) {
-#pragma unroll 1
-            for (int i = 0; i < kNBP; ++i) J += (S->bp[i] < r.x[j]);
+#pragma unroll
+            for (int step = 16; step; step >>= 1)          // number of breakpoints below x (sorted list)
+                if (J + step <= kNBP && S->bp[J + step - 1] < r.x[j]) J += step;
             const double2 pq = S->PQ[J];
             const double xd = (double)r.x[j], id = (double)r.I[j];
             const double d0 = __dsub_rn(xd, pq.x), d1 = __dsub_rn(xd, pq.y);
