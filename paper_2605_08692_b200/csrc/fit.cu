@@ -51,7 +51,7 @@
 // blocks as contiguous ranges (slab-major), so every sum has a fixed order and results are
 // bitwise reproducible.  A warp takes 4 rows; each lane 8 adjacent columns (one 128-bit load
 // per row), so its eight importances stay in registers.  A group is 2 lanes (g = 16) or 16
-// lanes (g = 128).  The next item's rows are loaded while the current item is processed.
+// lanes (g = 128).  A row's registers are refilled from the next item right after the row is unpacked.
 #include "lookup.cuh"
 
 namespace aaac {
@@ -142,24 +142,21 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     const int it0 = blockIdx.x * p.per_block;
     const int it1 = min(p.items, it0 + p.per_block);
 
-    uint4 nv[R];
-    uint32_t ns[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
-    auto load_item = [&](int slab, int rb) {
+    // Row registers of the item being processed; a row's registers are refilled with the same row
+    // of the next item as soon as the row has been unpacked, so the load has about an item's time
+    // to arrive and no second buffer is needed.
+    uint4 v[R];
+    uint32_t sc[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
+    auto load_row = [&](int u, int slab, int rb) {
         const int col0 = slab * 256 + lane * 8;
-        const int row0 = rb * kRowsPerItem + warp * R;
-        const uint16_t* wp = p.W + (size_t)row0 * (size_t)p.ldw + col0;
-        const uint32_t g0 = (uint32_t)col0 / G;
-#pragma unroll
-        for (int u = 0; u < R; ++u) {
-            const int row = row0 + u;
-            nv[u] = make_uint4(0, 0, 0, 0);
-            ns[u] = 0u;
-            if (col0 < K && row < N) {
-                nv[u] = __ldcs(reinterpret_cast<const uint4*>(wp + (size_t)u * (size_t)p.ldw));
-                const size_t gi = (size_t)row * (size_t)Gr + g0;
-                if (MODE == AAAC_NVFP4) ns[u] = p.scales[gi];      // masked at use: nothing waits on the load here
-                else ns[u] = __float_as_uint(__ldg(p.rinv + gi));
-            }
+        const int row = rb * kRowsPerItem + warp * R + u;
+        v[u] = make_uint4(0, 0, 0, 0);
+        sc[u] = 0u;
+        if (col0 < K && row < N) {
+            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
+            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+            if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];          // masked at use: nothing waits on the load here
+            else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
         }
     };
 
@@ -193,16 +190,15 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     // (slab, row block) of the current item and of the one being loaded
     int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
     int nslab = slab, nrb = rb;
-    if (it0 < it1) load_item(slab, rb);
-    for (int item = it0; item < it1; ++item) {
-        uint4 v[R];
-        uint32_t sc[R];
+    if (it0 < it1) {
 #pragma unroll
-        for (int u = 0; u < R; ++u) { v[u] = nv[u]; sc[u] = ns[u]; }
+        for (int u = 0; u < R; ++u) load_row(u, slab, rb);
+    }
+    for (int item = it0; item < it1; ++item) {
         slab = nslab;
         rb = nrb;
         if (++nrb == p.nrb) { nrb = 0; ++nslab; }
-        if (item + 1 < it1) load_item(nslab, nrb);
+        const bool more = item + 1 < it1;
 
         if (slab != cur_slab) {
             cur_slab = slab;
@@ -247,6 +243,11 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) & kBinMask;
                 e1v[j] = lds_table_u2(lut1_lane + off);
             }
+        };
+        // same, then refill the row's registers from the next item
+        auto L1n = [&](int u) {
+            L1(u);
+            if (more) load_row(u, nslab, nrb);
         };
         auto L2 = [&]() {
 #pragma unroll
@@ -316,13 +317,13 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
 
         if (nrows == R) {
             // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
-            L1(0);
+            L1n(0);
             L2();
             M(0, mt[0], ba[0]);
 #pragma unroll
             for (int u = 1; u < R; ++u) {
                 const int prev = (u - 1) & 1, cur = u & 1;
-                L1(u);
+                L1n(u);
                 B(mt[prev], ba[prev], 0, 4);
                 L2();
                 B(mt[prev], ba[prev], 4, 8);
@@ -330,20 +331,24 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             }
             B(mt[(R - 1) & 1], ba[(R - 1) & 1], 0, 8);
         } else {
-            // ragged last row block of the layer: row by row
-            for (int u = 0; u < nrows; ++u) {
-                // (u is uniform over the warp; the stages index v[] and sc[] with it)
-                uint4 vv = v[0];
-                uint32_t ss = sc[0];
+            // ragged last row block of the layer: row by row, then refill all rows
+            uint4 vr[R];
+            uint32_t sr[R];
 #pragma unroll
-                for (int t = 1; t < R; ++t)
-                    if (u == t) { vv = v[t]; ss = sc[t]; }
-                v[0] = vv;
-                sc[0] = ss;
+            for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; }
+            for (int u = 0; u < nrows; ++u) {
+                // (u is uniform over the warp; the stages read row 0 of v[] and sc[])
+#pragma unroll
+                for (int t = 0; t < R; ++t)
+                    if (u == t) { v[0] = vr[t]; sc[0] = sr[t]; }
                 L1(0);
                 L2();
                 M(0, mt[0], ba[0]);
                 B(mt[0], ba[0], 0, 8);
+            }
+            if (more) {
+#pragma unroll
+                for (int t = 0; t < R; ++t) load_row(t, nslab, nrb);
             }
         }
         Eacc += (double)eitem;

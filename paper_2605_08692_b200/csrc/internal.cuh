@@ -18,7 +18,7 @@ constexpr int kActMaxSplits = 256;
 
 // shape of the fit-round kernel: warps per block, copies of the {J_low, thr} table
 #ifndef AAAC_FIT_WARPS
-#define AAAC_FIT_WARPS 12
+#define AAAC_FIT_WARPS 16
 #endif
 #ifndef AAAC_FIT_REP
 #define AAAC_FIT_REP 8
