@@ -22,14 +22,15 @@
 //     whose entries are NaN: the group falls through to the exact path below, which searches J
 //     directly.
 // (b) Selection.  A second table gives {P, Q}: the FP32 roundings of the nearest entries of T0
-//     and T1 on interval J, with the low 4 mantissa bits replaced by the entry's index (so the
+//     and T1 on interval J, moved by at most 8 units in the last place so that the low 4 mantissa
+//     bits equal the entry's index (so the
 //     same 8 bytes also say which cell the weight falls into).  u_r = x - T_r,
 //     E_r = sum_k I_k u_r^2 (Eq. 8), summed per lane and over the lanes of the group by shuffles;
 //     sigma = [E1 < E0].
-//     Rounding: the constants differ from the entries by at most eta = 2^-19 max|T|, so
+//     Rounding: the constants differ from the entries by at most eta = 17 * 2^-24 max|T|, so
 //     |E_r - E_r,exact| <= 2^-24 * 16 E_r + 2 eta sum I |u_r| and
 //     sum I |u_r| <= sqrt(sum I * E_r).  Groups with
-//     |E0 - E1| <= 2^-24 (16 (E0 + E1) + 2.83 * 32 max|T| sqrt(sum I (E0 + E1))) (and NaN) are
+//     |E0 - E1| <= 2^-24 (16 (E0 + E1) + 2.83 * 17 max|T| sqrt(sum I (E0 + E1))) (and NaN) are
 //     re-evaluated in double with the exact entries, so sigma is the double-precision decision
 //     (the kernel tests against the slightly larger bound that sqrt(a b) <= a / 16 + 4 b gives,
 //     which needs one multiply-add per group).  The two errors are carried as one packed
@@ -83,6 +84,7 @@ __device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
     lo = __fadd_rn(lo, err);
 }
 
+constexpr int kMaxFitBlocks = 192;                    // grid limit: the partials of all blocks are staged in shared memory
 constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
 
 // Grid-wide barrier of a cooperative launch: block arrivals are counted in ctrl->bar, which only
@@ -389,13 +391,23 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         return;
     }
     {
+        // stage every block's partial in shared memory (the bins' space; all loads independent),
+        // then add them per value in kStrands interleaved strands, each in block order
+        static_assert((size_t)NW * kBinBytes >= (size_t)kMaxFitBlocks * kUsed * sizeof(float2), "staging space");
+        float2* stage = reinterpret_cast<float2*>(dyn + kLut1Bytes + kLut2Bytes);      // [grid][kUsed]
+        const int total = (int)gridDim.x * kUsed;
+#pragma unroll 8
+        for (int i = tid; i < total; i += NT) {
+            const int b = i / kUsed;
+            stage[i] = __ldcg(part + (size_t)b * kPartStride + (i - b * kUsed));
+        }
+        __syncthreads();
         constexpr int kStrands = NT / kUsed;
         const int strand = tid / kUsed, val = tid - strand * kUsed;
         if (strand < kStrands) {
             float hi = 0.f, lo = 0.f;
-#pragma unroll 4
-            for (unsigned b = strand; b < gridDim.x; b += kStrands) {
-                const float2 v = __ldcg(part + (size_t)b * kPartStride + val);
+            for (int b = strand; b < (int)gridDim.x; b += kStrands) {
+                const float2 v = stage[b * kUsed + val];
                 two_sum(hi, lo, v.x);
                 lo = __fadd_rn(lo, v.y);
             }
@@ -462,7 +474,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     if (N > 0x7FFFFFFF || K > 0x7FFFFFFF || items > 0x7FFFFFFF) return cudaErrorInvalidValue;
     int64_t grid = sm_count();
     if (grid > items) grid = items;
-    if (grid > kMaxBlocks) grid = kMaxBlocks;
+    if (grid > kMaxFitBlocks) grid = kMaxFitBlocks;
     const int64_t per_block = (items + grid - 1) / grid;
     grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;

@@ -83,7 +83,7 @@ struct FitTables {
     float rlut[128];              // NVFP4: fl32(1 / s_eff) per E4M3 code
     float2 pq32[kJSlots];         // {P, Q} of every interval before replication
     float centre[2 * kM];         // centre constant of every entry (index in the low 4 mantissa bits)
-    float tmax283;                // 2.83 * 32 * max |entry|, rounded up
+    float tmax283;                // 2.83 * 17 * max |entry|, rounded up
     int is_last;
     double tot[kPartStride];
 };
@@ -103,12 +103,18 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
     }
     if (tid >= 30 && tid < 32) S.bp[tid] = __int_as_float(0x7F800000);
     if (tid >= 32 && tid < 32 + 2 * kM) {
-        // centre constant: FP32 rounding of the entry with its canonical (lowest duplicate) index
-        // in the low mantissa bits
+        // centre constant: close to the FP32 rounding of the entry, with the entry's canonical
+        // (lowest duplicate) index in the low mantissa bits
         const int t = tid - 32, r = t & 16;
         int i = t & 15;
         while (i > 0 && S.Td[r + i - 1] == S.Td[r + i]) --i;
-        S.centre[t] = __uint_as_float((__float_as_uint((float)S.Td[t]) & ~kIdxMask) | (uint32_t)i);
+        // the float nearest to the FP32 rounding of the entry whose low 4 mantissa bits are i
+        // (at most 8 units in the last place away)
+        const uint32_t b = __float_as_uint((float)S.Td[t]);
+        const int mag = (int)(b & 0x7FFFFFFFu);
+        const int tt = mag + 8 - i;
+        const uint32_t mag2 = tt < 0 ? (uint32_t)i : (uint32_t)((tt & ~15) + i);
+        S.centre[t] = __uint_as_float((b & 0x80000000u) | mag2);
     }
     __syncthreads();
     if (tid < kNBP) {
@@ -124,8 +130,9 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
     if (tid < kJSlots) {
         float P = __int_as_float(0x7FC00000), Q = P;
         if (tid < kNJ) {
-            int i0 = 0, i1 = 0;
-            for (int j = 0; j < tid; ++j) { i0 += (S.src[j] == 0); i1 += (S.src[j] == 1); }
+            // entries of T0 / T1 whose upper midpoint lies below interval tid
+            const unsigned from1 = __ballot_sync(0x7FFFFFFFu, tid < kNBP && S.src[tid] == 1);
+            int i1 = __popc(from1 & ((1u << tid) - 1u)), i0 = tid - i1;
             while (i0 > 0 && S.Td[i0 - 1] == S.Td[i0]) --i0;
             while (i1 > 0 && S.Td[kM + i1 - 1] == S.Td[kM + i1]) --i1;
             S.PQ[tid] = make_double2(S.Td[i0], S.Td[kM + i1]);
@@ -137,7 +144,7 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
         double tm = fabs(S.Td[tid]);                     // 32 entries, one per lane of warp 0
 #pragma unroll
         for (int o = 16; o; o >>= 1) tm = fmax(tm, __shfl_xor_sync(0xFFFFFFFFu, tm, o));
-        if (tid == 0) S.tmax283 = __double2float_ru(tm * (2.83 * 32.0));
+        if (tid == 0) S.tmax283 = __double2float_ru(tm * (2.83 * 17.0));
         S.pq32[tid] = make_float2(P, Q);
     }
     // {J_low, thr} per bin.  Bin b holds the x with 64 x + 512 in [b - h, b + 1 - h], h = half of

@@ -8,7 +8,7 @@
 // lookup returns) and sigma into the sign bit of the scale.
 //
 // Exactness.  The group errors are summed in FP32 with constants that differ from the entries by
-// at most 2^-19 max|T|; groups inside the resulting error bound (see fit.cu) are re-evaluated in
+// at most 17 * 2^-24 max|T|; groups inside the resulting error bound (see fit.cu) are re-evaluated in
 // double with the exact entries, so sigma equals the double-precision decision.  The interval
 // search itself is exact (rounded-down midpoints), hence so are the codes.
 //
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
             for (int j = 0; j < 8; ++j) {
                 const uint32_t cb = __float_as_uint(sg ? pq[j].y : pq[j].x);
                 word |= (cb & kIdxMask) << (4 * j);
-                const float tv = __uint_as_float(cb & ~kIdxMask);          // the BF16 entry itself
+                const float tv = __uint_as_float((cb + 0x8000u) & 0xFFFF0000u);   // the BF16 entry itself (c is within 8 ulp of it)
                 const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
                 const float dw = __fmaf_rn(-tv, sval, wf);
                 eo = __fmaf_rn(__fmul_rn(Iv[j], dw), dw, eo);
