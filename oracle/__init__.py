@@ -125,6 +125,51 @@ def fit_round(wt, I, g, T01, want_sigma=False):
     return (T, E.value, sig) if want_sigma else (T, E.value)
 
 
+def assign(wt, I, g, T01):
+    """Assignment step alone (Alg. 1 lines 7-11).  Returns (sigma uint8 [N x K/g], objective)."""
+    wt = np.ascontiguousarray(wt, dtype=np.float32)
+    I = np.ascontiguousarray(I, dtype=np.float32)
+    N, K = wt.shape
+    T = np.ascontiguousarray(T01, dtype=np.float64).reshape(2, M)
+    sig = np.empty((N, K // g), dtype=np.uint8)
+    E = C.c_double(0.0)
+    rc = lib().oracle_assign(_p(wt), _p(I), C.c_int64(N), C.c_int64(K), C.c_int(g), _p(T), _p(sig), C.byref(E))
+    if rc:
+        raise ValueError(f"oracle_assign failed: {rc}")
+    return sig, E.value
+
+
+def inner_update(wt, I, g, sigma, T01) -> np.ndarray:
+    """One inner k-means iteration with sigma frozen (Alg. 1 lines 15-20), unsorted result."""
+    wt = np.ascontiguousarray(wt, dtype=np.float32)
+    I = np.ascontiguousarray(I, dtype=np.float32)
+    N, K = wt.shape
+    T = np.array(T01, dtype=np.float64).reshape(2, M).copy()
+    sig = np.ascontiguousarray(sigma, dtype=np.uint8)
+    assert sig.shape == (N, K // g)
+    rc = lib().oracle_inner_update(_p(wt), _p(I), _p(sig), C.c_int64(N), C.c_int64(K), C.c_int(g), _p(T))
+    if rc:
+        raise ValueError(f"oracle_inner_update failed: {rc}")
+    return T
+
+
+def sort_tables(T01) -> np.ndarray:
+    T = np.array(T01, dtype=np.float64).reshape(2, M).copy()
+    lib().oracle_sort_tables(_p(T))
+    return T
+
+
+def outer_iteration(wt, I, g, T01, n_inner):
+    """One pass of Alg. 1's outer loop in the paper's order: assignment step, then n_inner inner
+    iterations of each table with the selection frozen, then the sort.  Returns (new tables,
+    objective of the assignment step, sigma)."""
+    sig, E = assign(wt, I, g, T01)
+    T = np.array(T01, dtype=np.float64).reshape(2, M).copy()
+    for _ in range(n_inner):
+        T = inner_update(wt, I, g, sig, T)
+    return sort_tables(T), E, sig
+
+
 def objective(wt, I, g, T01) -> float:
     wt = np.ascontiguousarray(wt, dtype=np.float32)
     I = np.ascontiguousarray(I, dtype=np.float32)
@@ -184,8 +229,8 @@ def output_error(W, codes, s, ts, Tb, I, mode, g) -> float:
                                            C.c_int64(N), C.c_int64(K), C.c_int(mode), C.c_int(g)))
 
 
-def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=None):
-    """Algorithm 1 for one layer with n_inner = 1.
+def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=None, n_inner=1):
+    """Algorithm 1 for one layer (rounds = n_outer).
 
     Returns a dict: I, scales (sign bit = sigma), tensor_scale, T (float64 tables after the
     last round), T_f32, T_bf16, codes, sigma, trace (objective of each round's assignment
@@ -204,7 +249,10 @@ def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=Non
     T_start = T.copy()
     trace = []
     for _ in range(rounds):
-        T, E = fit_round(wt, I, g, T)
+        if n_inner == 1:
+            T, E = fit_round(wt, I, g, T)
+        else:
+            T, E, _ = outer_iteration(wt, I, g, T, n_inner)
         trace.append(E)
     Tf, Tb = round_tables(T)
     codes, sig, E_final, ties = pack(wt, I, g, Tb)

@@ -14,6 +14,9 @@
  *   oracle_init_grid      Sec. 3.1         the format's fixed table (INT4 grid / E2M1)
  *   oracle_fit_round      Alg. 1 lines 6-16 with n_inner = 1: assignment (Eq. 8),
  *                         weighted centroids (Eq. 11), keep-if-empty, sort
+ *   oracle_assign         Alg. 1 lines 7-11  assignment step alone: sigma per group, objective
+ *   oracle_inner_update   Alg. 1 lines 15-20 one inner k-means iteration with sigma frozen (no sort)
+ *   oracle_sort_tables    Alg. 1 line 22     ascending sort of each table
  *   oracle_objective      Eq. 8 summed over all groups (no update)
  *   oracle_round_tables   Alg. 1 line 17   round tables to BF16
  *   oracle_pack           Alg. 1 lines 18-19, Eq. 6
@@ -36,7 +39,10 @@
  *     s_t = layer absmax / (448 * 6)                       [parity unpinned]
  *   - quantile = linear interpolation at q (n - 1)         [parity unpinned]
  *   - nibble order: element 2i -> low nibble of byte i     [parity unpinned]
- *   - argmin ties: lowest index; sigma tie: table 0
+ *   - argmin ties: of two equidistant entries the smaller one, of equal entries the lowest
+ *     index (on an ascending table: the lowest index); sigma tie: table 0
+ *   - an inner iteration (Alg. 1 lines 15-20) updates all entries of a table at once, from
+ *     the cells of the table as it stood before the iteration (ordinary Lloyd / k-means)
  */
 #include <float.h>
 #include <math.h>
@@ -232,13 +238,16 @@ void oracle_init_grid(int mode, double* T01) {
 
 /* ------------------------------------------------------------ Eq. 4 */
 
-/* index of the nearest entry; the lowest index wins ties */
+/* index of the nearest entry; of two equidistant entries the smaller wins, of equal entries
+ * the lowest index (tables are ascending except between the inner iterations of one table
+ * update, where Alg. 1 sorts only after the last one; on an ascending table this is "the
+ * lowest index wins") */
 static int nearest(const double* T, double x) {
     int best = 0;
     double bd = fabs(x - T[0]);
     for (int i = 1; i < M; ++i) {
         double d = fabs(x - T[i]);
-        if (d < bd) { bd = d; best = i; }
+        if (d < bd || (d == bd && T[i] < T[best])) { bd = d; best = i; }
     }
     return best;
 }
@@ -311,6 +320,68 @@ int oracle_fit_round(const float* wt, const float* I, int64_t N, int64_t K, int 
     }
     if (E_out) *E_out = tot[4 * M];
     return OK;
+}
+
+/* Assignment step alone (Alg. 1 lines 7-11): sigma[N*K/g] and the Eq. 8 objective. */
+int oracle_assign(const float* wt, const float* I, int64_t N, int64_t K, int g,
+                  const double* T01, uint8_t* sigma, double* E_out) {
+    if (g > 128 || K % g) return ERR_ARG;
+    int64_t G = K / g;
+    double* rowE = (double*)calloc((size_t)N, sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        int idx[128];
+        for (int64_t j = 0; j < G; ++j) {
+            double E0, E1;
+            sigma[n * G + j] = (uint8_t)assign_group(wt + n * K + j * g, I + j * g, g, T01, &E0, &E1, idx);
+            rowE[n] += (E1 < E0) ? E1 : E0;
+        }
+    }
+    double E = 0.0;
+    for (int64_t n = 0; n < N; ++n) E += rowE[n];
+    free(rowE);
+    if (E_out) *E_out = E;
+    return OK;
+}
+
+/* One inner iteration of the table update (Alg. 1 lines 15-20) with the selection frozen:
+ * for r in {0, 1}, over the weights of the groups with sigma = r, every entry of T_r becomes the
+ * activation-weighted centroid (Eq. 11) of its Voronoi cell under T_r as it stood on entry;
+ * an entry whose denominator is zero keeps its value.  No sort (Alg. 1 sorts after the last
+ * inner iteration only). */
+int oracle_inner_update(const float* wt, const float* I, const uint8_t* sigma, int64_t N, int64_t K, int g,
+                        double* T01) {
+    if (g > 128 || K % g) return ERR_ARG;
+    int64_t G = K / g;
+    const int P = 2 * M * 2;
+    double* part = (double*)calloc((size_t)N * P, sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        double* p = part + n * P;                           /* [2][M] S, [2][M] Wt */
+        for (int64_t j = 0; j < G; ++j) {
+            const int r = sigma[n * G + j] ? 1 : 0;
+            for (int k = 0; k < g; ++k) {
+                const double x = (double)wt[n * K + j * g + k], imp = (double)I[j * g + k];
+                const int i = nearest(T01 + r * M, x);
+                p[r * M + i] += imp * x;
+                p[2 * M + r * M + i] += imp;
+            }
+        }
+    }
+    double tot[2 * M * 2];
+    for (int i = 0; i < P; ++i) tot[i] = 0.0;
+    for (int64_t n = 0; n < N; ++n)
+        for (int i = 0; i < P; ++i) tot[i] += part[n * P + i];
+    free(part);
+    for (int i = 0; i < 2 * M; ++i)
+        if (tot[2 * M + i] > 0.0) T01[i] = tot[i] / tot[2 * M + i];
+    return OK;
+}
+
+/* Alg. 1 line 22 */
+void oracle_sort_tables(double* T01) {
+    sort16(T01);
+    sort16(T01 + M);
 }
 
 /* sum over all groups of min_r (Eq. 8 error) for the given tables, no update */
