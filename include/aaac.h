@@ -44,7 +44,7 @@ typedef enum {
     AAAC_ERR_WORKSPACE = 5,     /* ws_bytes too small */
     AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
     AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
-    AAAC_ERR_UNIMPLEMENTED = 8, /* n_inner != 1 */
+    AAAC_ERR_UNIMPLEMENTED = 8, /* reserved */
     AAAC_ERR_TOO_LARGE = 9      /* size beyond the fixed capacity of a no-allocation entry point */
 } aaac_status;
 
@@ -104,8 +104,12 @@ int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64_t ldx, flo
  * Algorithm 1 lines 1-16 for one layer: scales (line 1), normalisation w~ = w / s (Eq. 2,
  * line 2; w~ = fl32(w * fl32(1/s)) is recomputed on the fly, never stored), importance
  * (line 3; taken from I, or computed from X when I == NULL), initial tables (lines 4-5),
- * then n_outer rounds of { assignment step Eq. 8, weighted-centroid update Eq. 11 with
- * n_inner = 1, keep an entry whose cell has no weight, sort }.
+ * then n_outer rounds of { assignment step Eq. 8; n_inner iterations of the weighted-centroid
+ * update Eq. 11 with the selection frozen, each from the Voronoi cells of the table as it stood
+ * before the iteration, an entry whose cell has no weight keeping its value; sort }.  With
+ * n_inner = 1 a round is a single pass over W (the cells of the update are the nearest-entry
+ * indices of the assignment step); every further inner iteration is one more, cheaper pass.
+ * n_inner >= 1 and n_outer * n_inner <= 2^20, else AAAC_ERR_SHAPE.
  *
  *   scales        out  positive scales (sign bit clear).  INT4: s = bf16(absmax/7) (1 for an
  *                      all-zero group).  NVFP4: E4M3(absmax / (6 s_t)) in 0x01..0x7E with

@@ -149,7 +149,7 @@ def timing_end(capacity: int):
 
 # ---- convenience for tests and the benchmark: allocate outputs, run the whole path ----
 
-def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trace=False, T01_init=None):
+def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trace=False, T01_init=None, n_inner=1):
     """Runs aaac_fit_layer then aaac_pack on device tensors and returns a dict of device tensors."""
     N, K = W.shape
     g = group_of(mode)
@@ -167,7 +167,7 @@ def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trac
         I = torch.empty(K, dtype=torch.float32, device=dev)
         act_stats(X, I, ws, dev_status=status)
     fit_layer(W, mode, I=I, n_outer=n_outer, init=init, T01=T01, scales=scales, tensor_scale=ts, ws=ws,
-              err_trace=trace, dev_status=status)
+              err_trace=trace, dev_status=status, n_inner=n_inner)
     T01_fit = T01.clone()
     scales_pos = scales.clone()
     Tb = torch.empty(2, 16, dtype=torch.uint16, device=dev)

@@ -89,7 +89,7 @@ const char* aaac_status_string(int status) {
         case AAAC_ERR_WORKSPACE: return "workspace too small";
         case AAAC_ERR_CUDA: return "CUDA runtime call or kernel launch failed";
         case AAAC_ERR_NONFINITE: return "input holds Inf or NaN";
-        case AAAC_ERR_UNIMPLEMENTED: return "not implemented (n_inner must be 1)";
+        case AAAC_ERR_UNIMPLEMENTED: return "not implemented";
         case AAAC_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this no-allocation entry point";
         default: return "unknown status";
     }
@@ -125,7 +125,7 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
     if (!I && !X) return AAAC_ERR_NULL;
     if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID && init != AAAC_INIT_USER) return AAAC_ERR_MODE;
     if (n_outer < 0) return AAAC_ERR_SHAPE;
-    if (n_inner != 1) return AAAC_ERR_UNIMPLEMENTED;
+    if (n_inner < 1 || (int64_t)n_outer * n_inner > (1 << 20)) return AAAC_ERR_SHAPE;
     if (!I && (T < 1 || ldx < K || ldx % 8)) return AAAC_ERR_SHAPE;
     if (!I && !aligned(X, 16)) return AAAC_ERR_ALIGN;
     if (I && !aligned(I, 16)) return AAAC_ERR_ALIGN;
@@ -156,7 +156,7 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
             }
         }
         if (e0) cudaEventRecord(e0, st);
-        if (launch_fit_rounds(Wp, N, K, ldw, mode, scales, I, n_outer, err_trace, dev_status, w, st) != cudaSuccess)
+        if (launch_fit_rounds(Wp, N, K, ldw, mode, scales, I, n_outer, n_inner, err_trace, dev_status, w, st) != cudaSuccess)
             return AAAC_ERR_CUDA;
         if (e1) cudaEventRecord(e1, st);
     }

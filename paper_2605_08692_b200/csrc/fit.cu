@@ -53,6 +53,8 @@
 // bitwise reproducible.  A warp takes 4 rows; each lane 8 adjacent columns (one 128-bit load
 // per row), so its eight importances stay in registers.  A group is 2 lanes (g = 16) or 16
 // lanes (g = 128).  A row's registers are refilled from the next item right after the row is unpacked.
+#include <type_traits>
+
 #include "lookup.cuh"
 
 namespace aaac {
@@ -69,7 +71,9 @@ struct FitParams {
     double* part;                 // [2][kMaxBlocks][kPartStride]: partials of even / odd rounds
     double* err_trace;            // [n_rounds] or null
     uint32_t* dev_status;         // or null
-    int n_rounds;
+    uint32_t* sigw;               // [N][slabs]: selection bits of a row's 256-column slab, bit = lane (n_inner > 1)
+    int n_rounds;                 // passes over W: n_outer * n_inner
+    int n_inner;
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
 };
 
@@ -114,7 +118,9 @@ __device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
     return S.is_last != 0;
 }
 
-template <int MODE, int NW, int REP>
+// HAS_INNER = false is the n_inner = 1 kernel (every pass an assignment pass, nothing kept between
+// passes but the tables); HAS_INNER = true adds the passes with the selection frozen.
+template <int MODE, int NW, int REP, bool HAS_INNER>
 __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;
@@ -141,26 +147,9 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     // 32-bit index arithmetic throughout (N, K < 2^31); only the final element offsets are 64-bit
     const int N = (int)p.N, K = (int)p.K;
     const int Gr = K / G;
+    const int slabs = (K + 255) >> 8;
     const int it0 = blockIdx.x * p.per_block;
     const int it1 = min(p.items, it0 + p.per_block);
-
-    // Row registers of the item being processed; a row's registers are refilled with the same row
-    // of the next item as soon as the row has been unpacked, so the load has about an item's time
-    // to arrive and no second buffer is needed.
-    uint4 v[R];
-    uint32_t sc[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
-    auto load_row = [&](int u, int slab, int rb) {
-        const int col0 = slab * 256 + lane * 8;
-        const int row = rb * kRowsPerItem + warp * R + u;
-        v[u] = make_uint4(0, 0, 0, 0);
-        sc[u] = 0u;
-        if (col0 < K && row < N) {
-            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
-            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
-            if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];          // masked at use: nothing waits on the load here
-            else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
-        }
-    };
 
     if (tid < 2 * kM) S.Td[tid] = p.ctrl->T[tid];
     if (MODE == AAAC_NVFP4 && tid >= 64 && tid < 192) {
@@ -174,13 +163,41 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
     constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
 
+  // A pass is an assignment pass (selection, then the first inner iteration in the same sweep) or,
+  // with n_inner > 1, one of the n_inner - 1 further inner iterations with the selection frozen.
+  int inner_left = 0, outer = 0;
   for (int round = 0; round < p.n_rounds; ++round) {
+    const bool inner = HAS_INNER && inner_left > 0;
     build_tables<MODE, NW, REP>(S, dyn);
     for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
     // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
     // most g1 * (E0 + E1) + g2 * sum I, with kappa = 1/8 (about the usual |w~ - entry|)
     const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
     double Eacc = 0.0;
+
+   auto pass = [&](auto inner_tag) {
+    constexpr bool INNER = decltype(inner_tag)::value;
+    constexpr bool keep_sigma = HAS_INNER && !INNER;
+    // Row registers of the item being processed; a row's registers are refilled with the same row
+    // of the next item as soon as the row has been unpacked, so the load has about an item's time
+    // to arrive and no second buffer is needed.
+    uint4 v[R];
+    uint32_t sc[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
+    uint32_t sgw[R];          // inner iteration: the row's stored selection bits
+    auto load_row = [&](int u, int slab, int rb) {
+        const int col0 = slab * 256 + lane * 8;
+        const int row = rb * kRowsPerItem + warp * R + u;
+        v[u] = make_uint4(0, 0, 0, 0);
+        sc[u] = 0u;
+        if (INNER) sgw[u] = 0u;
+        if (col0 < K && row < N) {
+            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
+            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+            if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];          // masked at use: nothing waits on the load here
+            else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
+            if (INNER) sgw[u] = __ldcg(p.sigw + (size_t)row * (size_t)slabs + slab);
+        }
+    };
 
     int cur_slab = -1;
     uint64_t II[8];           // {I, I} of the lane's eight columns
@@ -236,7 +253,9 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         uint64_t pq[8];                                    // {P, Q}, packed
         float mt[2][8];                                    // chosen centred term I (x - c) of the rows in B / M
         uint32_t ba[2][8];                                 // its bin address
+        bool sg_row = false;                               // inner iteration: this lane's stored selection bit
         auto L1 = [&](int u) {
+            if (INNER) sg_row = (sgw[u] >> lane) & 1u;
             const float rinv = MODE == AAAC_NVFP4 ? S.rlut[sc[u] & 0x7Fu] : __uint_as_float(sc[u]);
             const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
@@ -256,7 +275,41 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             for (int j = 0; j < 8; ++j)
                 pq[j] = lds_table_b64(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
         };
-        auto M = [&](int u, float (&mt_o)[8], uint32_t (&ba_o)[8]) {
+        auto M = [&](int row, float (&mt_o)[8], uint32_t (&ba_o)[8]) {
+            if constexpr (INNER) {
+                // selection frozen: the centred term under the stored table only.  A poisoned
+                // slot shows as NaN; those lanes search their intervals directly.
+                const bool sg = sg_row;
+                float c[8], chk = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float cP, cQ;
+                    unpack2(pq[j], cP, cQ);
+                    c[j] = sg ? cQ : cP;
+                    mt_o[j] = __fmul_rn(lo2(II[j]), __fsub_rn(x[j], c[j]));
+                    chk += mt_o[j];
+                }
+                const bool bad = !(chk == chk);
+                if (__any_sync(0xFFFFFFFFu, bad)) {
+                    Row8 r;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); }
+                    const Exact8 ex = exact_groups<LPG>(&S, r, (int)bad);
+                    if (bad) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float cP, cQ;
+                            unpack2(lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes)), cP, cQ);
+                            c[j] = sg ? cQ : cP;
+                            mt_o[j] = __fmul_rn(lo2(II[j]), __fsub_rn(x[j], c[j]));
+                        }
+                    }
+                }
+                const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) ba_o[j] = base + (__float_as_uint(c[j]) & kIdxMask) * kSlotBytes;
+                return;
+            }
             uint64_t m[8];                                 // {I (x - P), I (x - Q)}
             uint64_t e01 = 0ull;
 #pragma unroll
@@ -296,6 +349,10 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 }
             }
             if (col_ok && (lane % LPG) == 0) eitem += emin;
+            if (keep_sigma) {
+                const unsigned bits = __ballot_sync(0xFFFFFFFFu, sg);
+                if (lane == 0) p.sigw[(size_t)row * (size_t)slabs + slab] = bits;
+            }
             // cell = entry index (low bits of the centre constant) under the chosen table
             const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
 #pragma unroll
@@ -321,7 +378,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
             L1n(0);
             L2();
-            M(0, mt[0], ba[0]);
+            M(row0, mt[0], ba[0]);
 #pragma unroll
             for (int u = 1; u < R; ++u) {
                 const int prev = (u - 1) & 1, cur = u & 1;
@@ -329,23 +386,23 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 B(mt[prev], ba[prev], 0, 4);
                 L2();
                 B(mt[prev], ba[prev], 4, 8);
-                M(u, mt[cur], ba[cur]);
+                M(row0 + u, mt[cur], ba[cur]);
             }
             B(mt[(R - 1) & 1], ba[(R - 1) & 1], 0, 8);
         } else {
             // ragged last row block of the layer: row by row, then refill all rows
             uint4 vr[R];
-            uint32_t sr[R];
+            uint32_t sr[R], gr[R];
 #pragma unroll
-            for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; }
+            for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; gr[t] = INNER ? sgw[t] : 0u; }
             for (int u = 0; u < nrows; ++u) {
                 // (u is uniform over the warp; the stages read row 0 of v[] and sc[])
 #pragma unroll
                 for (int t = 0; t < R; ++t)
-                    if (u == t) { v[0] = vr[t]; sc[0] = sr[t]; }
+                    if (u == t) { v[0] = vr[t]; sc[0] = sr[t]; if (INNER) sgw[0] = gr[t]; }
                 L1(0);
                 L2();
-                M(0, mt[0], ba[0]);
+                M(row0 + u, mt[0], ba[0]);
                 B(mt[0], ba[0], 0, 8);
             }
             if (more) {
@@ -354,6 +411,13 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             }
         }
         Eacc += (double)eitem;
+    }
+   };
+    if constexpr (HAS_INNER) {
+        if (inner) pass(std::true_type{});
+        else pass(std::false_type{});
+    } else {
+        pass(std::false_type{});
     }
 
     // ---- block partial: lane c of a warp adds the 32 lane-private values of cell c (in a
@@ -437,7 +501,10 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         for (int i = 0; i < kM; ++i) rank += (tn[i] < t) || (tn[i] == t && i < (tid & 15));
         S.Td[(tid & 16) + rank] = t;
     }
-    if (blockIdx.x == 0 && tid == 0 && p.err_trace) p.err_trace[round] = S.tot[2 * kCells];
+    // the trace holds the Eq. 8 objective of each assignment step
+    if (!inner && blockIdx.x == 0 && tid == 0 && p.err_trace) p.err_trace[outer] = S.tot[2 * kCells];
+    if (inner) --inner_left;
+    else { inner_left = HAS_INNER ? p.n_inner - 1 : 0; ++outer; }
     __syncthreads();
   }
     if (blockIdx.x == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
@@ -447,10 +514,10 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
     if (threadIdx.x < 2 * kM) T01[threadIdx.x] = (float)ctrl->T[threadIdx.x];
 }
 
-template <int MODE, int NW, int REP>
+template <int MODE, int NW, int REP, bool HAS_INNER>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)REP * kNBins * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
-    auto kern = fit_rounds_kernel<MODE, NW, REP>;
+    auto kern = fit_rounds_kernel<MODE, NW, REP, HAS_INNER>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&p};
@@ -461,13 +528,16 @@ cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
-                              const float* I, int n_rounds, double* err_trace, uint32_t* dev_status,
+                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st) {
-    if (n_rounds <= 0) return cudaSuccess;
+    if (n_outer <= 0) return cudaSuccess;
+    if (n_inner < 1 || (int64_t)n_outer * n_inner > 0x7FFFFFFF) return cudaErrorInvalidValue;
     FitParams p{};
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
     p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
-    p.ctrl = ws.ctrl; p.part = ws.part; p.err_trace = err_trace; p.dev_status = dev_status; p.n_rounds = n_rounds;
+    p.ctrl = ws.ctrl; p.part = ws.part; p.err_trace = err_trace; p.dev_status = dev_status;
+    p.n_rounds = n_outer * n_inner; p.n_inner = n_inner;
+    p.sigw = ws.qlist;            // the quantile selection's list is free once the start tables exist
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
     const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
@@ -479,8 +549,12 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
-    if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP>(p, (unsigned)grid, st);
-    return launch_variant<AAAC_NVFP4, NW, REP>(p, (unsigned)grid, st);
+    if (n_inner > 1) {
+        if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, true>(p, (unsigned)grid, st);
+        return launch_variant<AAAC_NVFP4, NW, REP, true>(p, (unsigned)grid, st);
+    }
+    if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, false>(p, (unsigned)grid, st);
+    return launch_variant<AAAC_NVFP4, NW, REP, false>(p, (unsigned)grid, st);
 }
 
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st) {

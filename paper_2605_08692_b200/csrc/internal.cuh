@@ -56,7 +56,7 @@ struct Workspace {
     uint32_t* qhist;         // [kQBins]
     unsigned long long* qprefix;   // [kQBins + 1]
     uint8_t* qslot_of_bin;   // [kQBins]
-    uint32_t* qlist;         // [N*K]
+    uint32_t* qlist;         // [N*K]  candidates of the quantile selection; afterwards the fit's selection bits [N][ceil(K/256)]
     size_t bytes;
 };
 
@@ -97,7 +97,7 @@ cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, 
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
                         const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
-                              const float* I, int n_rounds, double* err_trace, uint32_t* dev_status,
+                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st);
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,

@@ -69,7 +69,8 @@ def test_argument_validation_happens_on_the_host(L):
     assert fit(n_outer=-1) == 3
     assert fit(init=9) == 2
     assert fit(W=odd) == 4
-    assert fit(n_inner=10) == 8
+    assert fit(n_inner=0) == 3
+    assert fit(n_outer=1 << 16, n_inner=1 << 8) == 3
     assert fit(I=None) == 1
     assert fit(wsb=C.c_size_t(1024)) == 5
     assert fit(ws=P((1 << 20) + 64)) == 4

@@ -85,11 +85,12 @@ def test_act_stats_strided_and_nonfinite():
 
 # ------------------------------------------------------------------ a2 scales, a3 init
 
-def run_fit(W, mode, I, rounds, init, want_trace=True, T01_init=None):
+def run_fit(W, mode, I, rounds, init, want_trace=True, T01_init=None, n_inner=1):
     Wd = dev_bf16(W)
     Id = torch.from_numpy(np.ascontiguousarray(I)).to(DEV)
     t0 = None if T01_init is None else torch.from_numpy(np.asarray(T01_init, dtype=np.float32)).to(DEV)
-    return binding.quantize_layer(Wd, mode, I=Id, n_outer=rounds, init=init, want_trace=want_trace, T01_init=t0)
+    return binding.quantize_layer(Wd, mode, I=Id, n_outer=rounds, init=init, want_trace=want_trace, T01_init=t0,
+                                  n_inner=n_inner)
 
 
 @pytest.mark.parametrize("mode", [INT4, NVFP4])
@@ -128,11 +129,11 @@ def test_user_tables_and_nonfinite_weights():
 
 # ------------------------------------------------------------------ a4-a6 fit rounds
 
-def check_fit(W, X, mode, rounds, init_name, rel_T=1e-5, rel_E=1e-4):
+def check_fit(W, X, mode, rounds, init_name, rel_T=1e-5, rel_E=1e-4, n_inner=1):
     g = 128 if mode == INT4 else 16
-    o = oracle.fit_layer(W, mode, g, rounds, X=X, init=init_name)
+    o = oracle.fit_layer(W, mode, g, rounds, X=X, init=init_name, n_inner=n_inner)
     init = dict(quantile=binding.INIT_QUANTILE, grid=binding.INIT_GRID)[init_name]
-    r = run_fit(W, mode, o["I"], rounds, init)
+    r = run_fit(W, mode, o["I"], rounds, init, n_inner=n_inner)
     ok, worst = table_close(host(r["T01"]), o["T"], rel_T)
     assert ok, f"tables differ: worst {worst:.3e}"
     if rounds:
@@ -271,6 +272,46 @@ def test_host_buffer_entry_point_matches_device_path():
     assert np.array_equal(err.numpy(), host(r["err"]))
     o = oracle.fit_layer(W, NVFP4, 16, 4, X=X)
     assert table_close(T01.numpy(), o["T"])[0]
+
+
+# ------------------------------------------------------------------ inner refinement (n_inner > 1)
+
+@pytest.mark.parametrize("mode,init", [(INT4, "grid"), (INT4, "quantile"), (NVFP4, "quantile")])
+@pytest.mark.parametrize("N,K,n_outer,n_inner", [(3, 256, 2, 2), (70, 640, 3, 4), (257, 1024, 3, 10)])
+def test_inner_refinement_small(mode, init, N, K, n_outer, n_inner):
+    """Algorithm 1 with n_inner > 1: ragged rows and columns, several items per block."""
+    W, X = layer(mode, N, K, name=f"inner{mode}{init}/{N}x{K}")
+    o, r, worst = check_fit(W, X, mode, n_outer, init, n_inner=n_inner)
+    check_pack(W, mode, o, r)
+    assert np.all(host(r["scales_pos"]) == o["scales_unsigned"])      # the fit leaves the scales' sign bits clear
+
+
+def test_inner_refinement_paper_budgets_full_size():
+    """The paper's default budget (n_outer, n_inner) = (3, 10) on the q_proj-sized layer of the
+    benchmark configuration, whole layer against the oracle, and n_inner = 1 through the same
+    entry point still equal to the single-pass rounds."""
+    c = synth.config2_layer("q_proj")
+    W, X = c["W"], c["X"]
+    o, r, worst = check_fit(W, X, NVFP4, 3, "quantile", n_inner=10)
+    check_pack(W, NVFP4, o, r)
+    print(f"(3,10): worst table deviation {worst:.2e}")
+    a = run_fit(W, NVFP4, o["I"], 3, binding.INIT_QUANTILE, n_inner=10)
+    assert torch.equal(a["T01"], r["T01"]) and torch.equal(a["codes"], r["codes"])   # reproducible
+
+
+def test_inner_refinement_degenerate_tables():
+    """Identical tables: every group ties (table 0), table 1 receives nothing in any inner
+    iteration and keeps its entries; entries of table 0 that coincide stay put."""
+    W, X = layer(INT4, 24, 256, name="innerdegen")
+    I = oracle.act_stats(X)
+    T0 = np.linspace(-6.5, 6.5, 16)
+    T0[7] = T0[6]                                        # a duplicate entry: its cell is empty
+    T = np.stack([T0, T0]).astype(np.float32)
+    o = oracle.fit_layer(W, INT4, 128, 2, I=I, init="user", T_init=T, n_inner=5)
+    r = run_fit(W, INT4, I, 2, binding.INIT_USER, T01_init=T, n_inner=5)
+    ok, worst = table_close(host(r["T01"]), o["T"])
+    assert ok, worst
+    assert np.allclose(host(r["trace"])[:2], o["trace"], rtol=1e-4)
 
 
 # ------------------------------------------------------------------ full benchmark sizes
