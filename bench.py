@@ -172,6 +172,9 @@ def run_stack(args, which):
     from paper_2605_08692_b200 import binding, build
     build.build()
     L, H, KV, FF, mode, tokens, rounds = STACKS[which]
+    n_inner = 1
+    if args.budget:                      # e.g. 3,10: the paper's default (n_outer, n_inner)
+        rounds, n_inner = (int(v) for v in args.budget.split(","))
     g = 128 if mode == 0 else 16
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -212,8 +215,8 @@ def run_stack(args, which):
             binding.act_stats(x, Iv[k], out["down" if k == "down" else "q"]["ws"], dev_status=status)
         for n, N, K, xin in lin:
             o = out[n]
-            binding.fit_layer(Ws[n], mode, I=Iv[xin], n_outer=rounds, init=binding.INIT_QUANTILE, T01=o["T01"],
-                              scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
+            binding.fit_layer(Ws[n], mode, I=Iv[xin], n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE,
+                              T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
             binding.pack(Ws[n], mode, I=Iv[xin], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"],
                          tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"])
 
@@ -236,9 +239,9 @@ def run_stack(args, which):
             "dtype": "f32", "data": "synthetic (device-generated, one decoder layer's tensors reused for every layer)",
             "config": {"workload": f"{which}: {L} decoder layers x 7 linears (hidden {H}, kv {KV}, intermediate {FF}), "
                                    f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'}, {tokens} tokens per input, quantile init, "
-                                   f"{rounds} rounds; act_stats + scales + init + rounds + pack",
-                       "linears": 7 * L, "weights": wl * L, "rounds": rounds},
-            "gweights_per_s_per_round": wl * L * rounds / wall / 1e9, "clocks": clocks}
+                                   f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds + pack",
+                       "linears": 7 * L, "weights": wl * L, "rounds": rounds, "n_inner": n_inner},
+            "gweights_per_s_per_round": wl * L * rounds * n_inner / wall / 1e9, "clocks": clocks}
     print(json.dumps(line), flush=True)
 
 
@@ -253,6 +256,8 @@ def main():
                     help="subset of the workload's layers (profiling a small case); the default is the full workload")
     ap.add_argument("--workload", default="cfg2", choices=["cfg2"] + sorted(STACKS),
                     help="cfg2 (default): the benchmark contract; stack8b / stack7b: wall time of a whole decoder stack")
+    ap.add_argument("--budget", default="",
+                    help="stack workloads only: n_outer,n_inner (default: the workload's rounds with n_inner = 1)")
     args = ap.parse_args()
     if args.workload != "cfg2":
         if int(os.environ.get("RANK", "0")) == 0:

@@ -1,10 +1,17 @@
-// The fit rounds (Algorithm 1 lines 6-16 with n_inner = 1): per round the assignment step
-// (Eq. 8) and the activation-weighted centroid update (Eq. 11) in a single pass over W.  All
+// The fit rounds (Algorithm 1 lines 6-16).  With n_inner = 1 a round is the assignment step
+// (Eq. 8) and the activation-weighted centroid update (Eq. 11) in a single pass over W, and all
 // rounds of a layer run in ONE persistent kernel (one block per SM, cooperative launch): after
 // its pass every block publishes a partial, the blocks meet at a grid-wide barrier, and every
 // block adds all partials in the same fixed order, so each holds the same new tables without a
 // second barrier or a relaunch.  The barrier wait is bounded: if it runs out, the kernel sets
 // AAAC_DEV_TIMEOUT in the device status word and returns.
+// With n_inner > 1 the assignment pass (which is also the first inner iteration) stores the
+// selection bits, one word per row and 256-column slab, and the remaining n_inner - 1 inner
+// iterations are passes of a second instance of the kernel that reads those bits instead of
+// forming the two errors; both instances share everything else.  The tables are put in
+// ascending order after every pass: in one dimension a centroid update keeps an ascending table
+// ascending (ties aside), and the cells depend on the entries' values only, so this equals
+// sorting after the last inner iteration.
 //
 // Per weight the kernel needs (a) the interval J of the merged breakpoint list of both tables
 // that holds w~ = fl32(w * r) (Eq. 2) -- J fixes the nearest entry of T0 and of T1 (Eq. 4) --
@@ -72,8 +79,9 @@ struct FitParams {
     double* err_trace;            // [n_rounds] or null
     uint32_t* dev_status;         // or null
     uint32_t* sigw;               // [N][slabs]: selection bits of a row's 256-column slab, bit = lane (n_inner > 1)
-    int n_rounds;                 // passes over W: n_outer * n_inner
-    int n_inner;
+    int n_rounds;                 // passes over W in this launch
+    int trace_base;               // err_trace index of this launch's first assignment pass
+    unsigned bar_base;            // passes of the layer's earlier launches (the barrier count keeps growing)
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
 };
 
@@ -118,9 +126,14 @@ __device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
     return S.is_last != 0;
 }
 
-// HAS_INNER = false is the n_inner = 1 kernel (every pass an assignment pass, nothing kept between
-// passes but the tables); HAS_INNER = true adds the passes with the selection frozen.
-template <int MODE, int NW, int REP, bool HAS_INNER>
+// A launch runs passes of one kind.  kRounds: assignment passes, each also the (only) inner
+// iteration of its round -- the n_inner = 1 procedure, all rounds of a layer in one launch.
+// kAssignKeep: the same pass, which also stores the selection bits.  kInner: further inner
+// iterations with the stored selection.  With n_inner > 1 a round is one kAssignKeep launch of a
+// single pass followed by one kInner launch of n_inner - 1 passes.
+enum PassKind { kRounds = 0, kAssignKeep = 1, kInner = 2 };
+
+template <int MODE, int NW, int REP, int KIND>
 __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;
@@ -163,11 +176,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
     constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
 
-  // A pass is an assignment pass (selection, then the first inner iteration in the same sweep) or,
-  // with n_inner > 1, one of the n_inner - 1 further inner iterations with the selection frozen.
-  int inner_left = 0, outer = 0;
   for (int round = 0; round < p.n_rounds; ++round) {
-    const bool inner = HAS_INNER && inner_left > 0;
     build_tables<MODE, NW, REP>(S, dyn);
     for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
     // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
@@ -177,7 +186,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
 
    auto pass = [&](auto inner_tag) {
     constexpr bool INNER = decltype(inner_tag)::value;
-    constexpr bool keep_sigma = HAS_INNER && !INNER;
+    constexpr bool keep_sigma = KIND == kAssignKeep;
     // Row registers of the item being processed; a row's registers are refilled with the same row
     // of the next item as soon as the row has been unpacked, so the load has about an item's time
     // to arrive and no second buffer is needed.
@@ -413,12 +422,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         Eacc += (double)eitem;
     }
    };
-    if constexpr (HAS_INNER) {
-        if (inner) pass(std::true_type{});
-        else pass(std::false_type{});
-    } else {
-        pass(std::false_type{});
-    }
+    pass(std::integral_constant<bool, KIND == kInner>{});
 
     // ---- block partial: lane c of a warp adds the 32 lane-private values of cell c (in a
     //      rotated, fixed order that avoids bank conflicts); then the warps are added ----
@@ -450,7 +454,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
 
     // ---- all blocks meet; then each adds the partials of all blocks in the same fixed order
     //      (kStrands interleaved strands per value, each in block order, then the strands) ----
-    if (!grid_barrier(S, p.ctrl, (unsigned)(round + 1) * gridDim.x)) {
+    if (!grid_barrier(S, p.ctrl, (p.bar_base + (unsigned)round + 1u) * gridDim.x)) {
         if (blockIdx.x == 0 && tid == 0 && p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
         return;
     }
@@ -502,9 +506,8 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         S.Td[(tid & 16) + rank] = t;
     }
     // the trace holds the Eq. 8 objective of each assignment step
-    if (!inner && blockIdx.x == 0 && tid == 0 && p.err_trace) p.err_trace[outer] = S.tot[2 * kCells];
-    if (inner) --inner_left;
-    else { inner_left = HAS_INNER ? p.n_inner - 1 : 0; ++outer; }
+    if (KIND != kInner && blockIdx.x == 0 && tid == 0 && p.err_trace)
+        p.err_trace[p.trace_base + round] = S.tot[2 * kCells];
     __syncthreads();
   }
     if (blockIdx.x == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
@@ -514,10 +517,10 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
     if (threadIdx.x < 2 * kM) T01[threadIdx.x] = (float)ctrl->T[threadIdx.x];
 }
 
-template <int MODE, int NW, int REP, bool HAS_INNER>
+template <int MODE, int NW, int REP, int KIND>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)REP * kNBins * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
-    auto kern = fit_rounds_kernel<MODE, NW, REP, HAS_INNER>;
+    auto kern = fit_rounds_kernel<MODE, NW, REP, KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&p};
@@ -536,7 +539,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
     p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
     p.ctrl = ws.ctrl; p.part = ws.part; p.err_trace = err_trace; p.dev_status = dev_status;
-    p.n_rounds = n_outer * n_inner; p.n_inner = n_inner;
+    p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
     p.sigw = ws.qlist;            // the quantile selection's list is free once the start tables exist
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
@@ -549,12 +552,23 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
-    if (n_inner > 1) {
-        if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, true>(p, (unsigned)grid, st);
-        return launch_variant<AAAC_NVFP4, NW, REP, true>(p, (unsigned)grid, st);
+    auto launch = [&](auto kind) {
+        constexpr int KIND = decltype(kind)::value;
+        if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, KIND>(p, (unsigned)grid, st);
+        return launch_variant<AAAC_NVFP4, NW, REP, KIND>(p, (unsigned)grid, st);
+    };
+    if (n_inner == 1) return launch(std::integral_constant<int, kRounds>{});
+    for (int outer = 0; outer < n_outer; ++outer) {
+        p.n_rounds = 1; p.trace_base = outer;
+        cudaError_t e = launch(std::integral_constant<int, kAssignKeep>{});
+        if (e != cudaSuccess) return e;
+        p.bar_base += 1u;
+        p.n_rounds = n_inner - 1;
+        e = launch(std::integral_constant<int, kInner>{});
+        if (e != cudaSuccess) return e;
+        p.bar_base += (unsigned)(n_inner - 1);
     }
-    if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, false>(p, (unsigned)grid, st);
-    return launch_variant<AAAC_NVFP4, NW, REP, false>(p, (unsigned)grid, st);
+    return cudaSuccess;
 }
 
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st) {
