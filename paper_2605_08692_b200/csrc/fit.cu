@@ -18,16 +18,18 @@
 // (b) its two weighted squared errors, and (c) one accumulation into the centroid sums of cell
 // (sigma, J).
 //
-// (a) Interval.  Uniform bins of width 1/64 on (-8, 8): the mantissa of
-//     fl32(64 x + 512 + 1.5 * 2^(23-k)) holds (64 x + 512) * 2^k rounded to an integer; masked,
+// (a) Interval.  NB uniform bins on (-8, 8) (512 of width 1/32 here; the pack pass, which has no
+//     bins to hold, uses 1024 of width 1/64): with s = NB / 16 the mantissa of
+//     fl32(s x + NB / 2 + 1.5 * 2^(23-k)) holds (s x + NB / 2) * 2^k rounded to an integer; masked,
 //     it is the byte offset bin * 2^k of the bin's table entry (2^k = bytes per bin over all
-//     copies), bin = floor of 64 x + 512 after rounding to a multiple of 2^-k.
+//     copies), bin = floor of s x + NB / 2 after rounding to a multiple of 2^-k.
 //     A table gives per bin {J_low, thr}: J_low breakpoints lie
 //     below the bin, thr is the one breakpoint inside it (+inf if none), J = J_low + (x > thr).
 //     Breakpoints are the rounded-down FP32 midpoints, for which x > thr <=> x > midpoint, so J
 //     is exact.  A bin that holds two or more breakpoints points at a poisoned slot (J = 31)
 //     whose entries are NaN: the group falls through to the exact path below, which searches J
-//     directly.
+//     directly.  (Fitted tables keep their merged breakpoints apart -- the two codebooks
+//     specialise -- so such bins are rare outside degenerate starts.)
 // (b) Selection.  A second table gives {P, Q}: the FP32 roundings of the nearest entries of T0
 //     and T1 on interval J, moved by at most 8 units in the last place so that the low 4 mantissa
 //     bits equal the entry's index (so the
@@ -51,9 +53,9 @@
 //     sorted; block 0 stores the Eq. 8 objective of the round (sum over groups of the smaller
 //     error) and, after the last round, the tables.
 //
-// Tables in shared memory are replicated to cut bank conflicts: the {J_low, thr} table REP
-// times (lane l uses copy l mod REP), the {P, Q} table and the bins once per lane (conflict
-// free).
+// Tables in shared memory are replicated against bank conflicts: the {J_low, thr} table REP = 16
+// times (lane l uses copy l mod 16, so the 16 lanes that share a wavefront of an 8-byte load
+// never collide), the {P, Q} table and the bins once per lane.
 //
 // Thread mapping.  A block of NW warps works on items of 4 NW rows x 256 columns, dealt to
 // blocks as contiguous ranges (slab-major), so every sum has a fixed order and results are
@@ -135,12 +137,13 @@ enum PassKind { kRounds = 0, kAssignKeep = 1, kInner = 2 };
 
 template <int MODE, int NW, int REP, int KIND>
 __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
+    constexpr int NB = AAAC_FIT_BINS;
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;
     constexpr int R = kRowsPerWarp;
     constexpr int kRowsPerItem = R * NW;
     constexpr int NT = NW * 32;
-    constexpr int kLut1Bytes = REP * kNBins * 8;
+    constexpr int kLut1Bytes = REP * NB * 8;
     constexpr int kLut2Bytes = kJSlots * kSlotBytes;
     constexpr int kBinBytes = kCells * kSlotBytes;           // per warp
     static_assert(kLut1Bytes >= NW * kPartStride * 8, "the per-warp partials reuse the first table's space");
@@ -172,12 +175,13 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     }
     __syncthreads();
 
-    // bin arithmetic: the masked mantissa of fl32(64 x + kMagic) is bin * (REP * 8)
-    constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
-    constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
+    // bin arithmetic: the masked mantissa of fl32(kBinsPerUnit x + kMagic) is bin * (REP * 8)
+    constexpr float kBinsPerUnit = (float)(NB / 16);
+    constexpr float kMagic = (float)(NB / 2) + 1.5f * (float)(1 << 23) / (float)(REP * 8);
+    constexpr uint32_t kBinMask = (uint32_t)(NB - 1) * (REP * 8);
 
   for (int round = 0; round < p.n_rounds; ++round) {
-    build_tables<MODE, NW, REP>(S, dyn);
+    build_tables<MODE, NW, REP, NB>(S, dyn);
     for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
     // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
     // most g1 * (E0 + E1) + g2 * sum I, with kappa = 1/8 (about the usual |w~ - entry|)
@@ -270,7 +274,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) & kBinMask;
+                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask;
                 e1v[j] = lds_table_u2(lut1_lane + off);
             }
         };
@@ -519,7 +523,7 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
 
 template <int MODE, int NW, int REP, int KIND>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
-    constexpr size_t smem = (size_t)REP * kNBins * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
+    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
     auto kern = fit_rounds_kernel<MODE, NW, REP, KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -21,7 +21,10 @@ constexpr int kActMaxSplits = 256;
 #define AAAC_FIT_WARPS 16
 #endif
 #ifndef AAAC_FIT_REP
-#define AAAC_FIT_REP 8
+#define AAAC_FIT_REP 16           // one copy per lane of a half-warp: an 8-byte lookup has no bank conflicts
+#endif
+#ifndef AAAC_FIT_BINS
+#define AAAC_FIT_BINS 512         // uniform bins of the {J_low, thr} table on (-8, 8): width 1/32
 #endif
 
 // ---- control block at the start of the workspace (device memory) ----

@@ -8,7 +8,7 @@
 namespace aaac {
 
 constexpr int kRowsPerWarp = 4;
-constexpr int kNBins = 1024;
+constexpr int kNBins = 1024;                       // default number of uniform bins on (-8, 8): width 1/64
 constexpr int kJSlots = 32;                        // 31 intervals + the poisoned slot
 constexpr int kSlotBytes = 32 * 8;                 // one 8-byte entry per lane
 constexpr int kPoison = kNJ * kSlotBytes;          // byte offset of the poisoned slot
@@ -89,7 +89,7 @@ struct FitTables {
 };
 
 // Builds every lookup table of the round from the current tables in S.Td.
-template <int MODE, int NW, int REP>
+template <int MODE, int NW, int REP, int NB = kNBins>
 __device__ void build_tables(FitTables& S, unsigned char* dyn) {
     constexpr int NT = NW * 32;
     const int tid = threadIdx.x;
@@ -126,7 +126,7 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
         S.exact[rank] = S.tmp_exact[tid];
     }
     __syncthreads();
-    float2* lut2 = reinterpret_cast<float2*>(dyn + (size_t)REP * kNBins * 8);
+    float2* lut2 = reinterpret_cast<float2*>(dyn + (size_t)REP * NB * 8);
     if (tid < kJSlots) {
         float P = __int_as_float(0x7FC00000), Q = P;
         if (tid < kNJ) {
@@ -147,13 +147,14 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
         if (tid == 0) S.tmax283 = __double2float_ru(tm * (2.83 * 17.0));
         S.pq32[tid] = make_float2(P, Q);
     }
-    // {J_low, thr} per bin.  Bin b holds the x with 64 x + 512 in [b - h, b + 1 - h], h = half of
-    // the rounding step 1 / (8 REP) of the bin arithmetic.  The breakpoints are sorted, so those
+    // {J_low, thr} per bin.  With s = NB / 16 bins per unit, bin b holds the x with s x + NB / 2 in
+    // [b - h, b + 1 - h], h = half of the rounding step 1 / (8 REP) of the bin arithmetic.  The breakpoints are sorted, so those
     // inside a bin are the first ones not below its lower edge.
     uint2* lut1 = reinterpret_cast<uint2*>(dyn);
     constexpr float h = 0.5f / (float)(REP * 8);
-    for (int b = tid; b < kNBins; b += NT) {
-        const float lo = ((float)b - 512.f - h) * 0.015625f, hi = ((float)b - 511.f - h) * 0.015625f;
+    constexpr float kHalf = (float)(NB / 2), kWidth = 16.f / (float)NB;
+    for (int b = tid; b < NB; b += NT) {
+        const float lo = ((float)b - kHalf - h) * kWidth, hi = ((float)b - (kHalf - 1.f) - h) * kWidth;
         int below = 0;                                   // number of breakpoints < lo (binary search)
 #pragma unroll
         for (int step = 16; step; step >>= 1)
