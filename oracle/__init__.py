@@ -46,6 +46,7 @@ def lib():
         _lib.oracle_e4m3_encode.restype = C.c_uint8
         _lib.oracle_e4m3_encode.argtypes = [C.c_float]
         _lib.oracle_max_threads.restype = C.c_int
+        _lib.oracle_output_error_sel.restype = C.c_double
     return _lib
 
 
@@ -229,8 +230,42 @@ def output_error(W, codes, s, ts, Tb, I, mode, g) -> float:
                                            C.c_int64(N), C.c_int64(K), C.c_int(mode), C.c_int(g)))
 
 
-def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=None, n_inner=1):
-    """Algorithm 1 for one layer (rounds = n_outer).
+def pack_sigma_bits(sigma) -> np.ndarray:
+    """Alg. 1 line 20 for S < g: sigma [N x K/S] -> bits uint8 [N x K/(8 S)], group j of a row in bit
+    j % 8 of byte j // 8."""
+    sig = np.ascontiguousarray(sigma, dtype=np.uint8)
+    N, GS = sig.shape
+    bits = np.empty((N, GS // 8), dtype=np.uint8)
+    rc = lib().oracle_pack_sigma_bits(_p(sig), C.c_int64(N), C.c_int64(GS), _p(bits))
+    if rc:
+        raise ValueError(f"oracle_pack_sigma_bits failed: {rc}")
+    return bits
+
+
+def dequant_sel(codes, s, ts, Tb, sigma_bits, S, mode, g) -> np.ndarray:
+    """Eq. 5 with separately stored selection bits (selection group S, scale group g)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    N, K = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((N, K), dtype=np.uint16)
+    lib().oracle_dequant_sel(_p(codes), _p(np.ascontiguousarray(s)), _p(ts), _p(_u16(Tb)),
+                             _p(np.ascontiguousarray(sigma_bits, dtype=np.uint8)), C.c_int(S), C.c_int64(N),
+                             C.c_int64(K), C.c_int(mode), C.c_int(g), _p(out), C.c_int64(K))
+    return out
+
+
+def output_error_sel(W, codes, s, ts, Tb, sigma_bits, S, I, mode, g) -> float:
+    W = _u16(W)
+    N, K = W.shape
+    return float(lib().oracle_output_error_sel(_p(W), C.c_int64(K), _p(np.ascontiguousarray(codes)),
+                                               _p(np.ascontiguousarray(s)), _p(ts), _p(_u16(Tb)),
+                                               _p(np.ascontiguousarray(sigma_bits, dtype=np.uint8)), C.c_int(S),
+                                               _p(np.ascontiguousarray(I, dtype=np.float32)),
+                                               C.c_int64(N), C.c_int64(K), C.c_int(mode), C.c_int(g)))
+
+
+def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=None, n_inner=1, S=None):
+    """Algorithm 1 for one layer (rounds = n_outer).  S = selection group size (default g); with
+    S < g the scales keep a clear sign bit and the selection bits come back as sigma_bits.
 
     Returns a dict: I, scales (sign bit = sigma), tensor_scale, T (float64 tables after the
     last round), T_f32, T_bf16, codes, sigma, trace (objective of each round's assignment
@@ -250,12 +285,16 @@ def fit_layer(W, mode, g, rounds, *, I=None, X=None, init="quantile", T_init=Non
     trace = []
     for _ in range(rounds):
         if n_inner == 1:
-            T, E = fit_round(wt, I, g, T)
+            T, E = fit_round(wt, I, S or g, T)
         else:
-            T, E, _ = outer_iteration(wt, I, g, T, n_inner)
+            T, E, _ = outer_iteration(wt, I, S or g, T, n_inner)
         trace.append(E)
     Tf, Tb = round_tables(T)
-    codes, sig, E_final, ties = pack(wt, I, g, Tb)
+    codes, sig, E_final, ties = pack(wt, I, S or g, Tb)
+    if S is not None and S != g:
+        return dict(I=I, scales=s, scales_unsigned=s, sigma_bits=pack_sigma_bits(sig), tensor_scale=ts, T=T,
+                    T_init=T_start, T_f32=Tf, T_bf16=Tb, codes=codes, sigma=sig, trace=np.array(trace),
+                    E_final=E_final, ties=ties, wt=wt)
     s_signed = apply_sigma(s, sig, mode)
     return dict(I=I, scales=s_signed, scales_unsigned=s, tensor_scale=ts, T=T, T_init=T_start, T_f32=Tf, T_bf16=Tb,
                 codes=codes, sigma=sig, trace=np.array(trace), E_final=E_final, ties=ties, wt=wt)

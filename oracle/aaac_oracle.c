@@ -22,6 +22,11 @@
  *   oracle_pack           Alg. 1 lines 18-19, Eq. 6
  *   oracle_apply_sigma    Alg. 1 line 20   selection bit -> sign bit of the scale
  *   oracle_dequant        Eq. 5
+ *   oracle_pack_sigma_bits, oracle_dequant_sel, oracle_output_error_sel
+ *                         the same with a selection group S smaller than the scale group g
+ *                         (Sec. 3.1 "granularity"): sigma stored apart, 1/S bit per weight.
+ *                         The fit and pack steps take the selection group size as their group
+ *                         argument: they see normalised weights only, so g does not enter them.
  *   oracle_output_error   Sec. 3.2 "Activation importance": sum_k I_k (w - w^)^2
  *
  * Arithmetic.  Everything is double except the quantities that are *defined* as
@@ -39,6 +44,8 @@
  *     s_t = layer absmax / (448 * 6)                       [parity unpinned]
  *   - quantile = linear interpolation at q (n - 1)         [parity unpinned]
  *   - nibble order: element 2i -> low nibble of byte i     [parity unpinned]
+ *   - separate selection bits (S < g): row-major, selection group j of a row in bit j mod 8 of
+ *     byte j / 8 of the row's K / (8 S) bytes                [parity unpinned]
  *   - argmin ties: of two equidistant entries the smaller one, of equal entries the lowest
  *     index (on an ascending table: the lowest index); sigma tie: table 0
  *   - an inner iteration (Alg. 1 lines 15-20) updates all entries of a table at once, from
@@ -511,6 +518,64 @@ double oracle_output_error(const uint16_t* W, int64_t ldw, const uint8_t* codes,
             int sigma = (mode == MODE_INT4) ? (((const uint16_t*)scales)[j] >> 15)
                                             : (((const uint8_t*)scales)[j] >> 7);
             double s = (double)scale_value(scales, j, mode, s_t);
+            int c = (e & 1) ? (codes[e >> 1] >> 4) : (codes[e >> 1] & 0x0F);
+            double d = (double)bf16_to_f32(W[n * ldw + k]) - (double)bf16_to_f32(Tb[sigma * M + c]) * s;
+            rowE += (double)I[k] * (d * d);
+        }
+        E += rowE;
+    }
+    return E;
+}
+
+/* ------------------------------------------------------------ S < g: selection bits apart */
+
+/* Alg. 1 line 20, S < g: the selection bits are stored separately, 1/S bit per weight.
+ * sigma [N][GS] (one byte per selection group) -> bits [N][GS / 8], group j of a row in
+ * bit j % 8 of the row's byte j / 8.  GS must be a multiple of 8. */
+int oracle_pack_sigma_bits(const uint8_t* sigma, int64_t N, int64_t GS, uint8_t* bits) {
+    if (GS % 8) return ERR_ARG;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t b = 0; b < GS / 8; ++b) {
+            unsigned v = 0;
+            for (int i = 0; i < 8; ++i) v |= (unsigned)(sigma[n * GS + b * 8 + i] ? 1 : 0) << i;
+            bits[n * (GS / 8) + b] = (uint8_t)v;
+        }
+    return OK;
+}
+
+static int sigma_bit(const uint8_t* bits, int64_t n, int64_t GS, int64_t j) {
+    return (bits[n * (GS / 8) + j / 8] >> (j % 8)) & 1;
+}
+
+/* Eq. 5 with sigma taken from the separate bits (selection group S) and the scale (sign bit
+ * clear) from its own group of g weights. */
+void oracle_dequant_sel(const uint8_t* codes, const void* scales, const float* tensor_scale,
+                        const uint16_t* Tb, const uint8_t* sigma_bits, int S, int64_t N, int64_t K,
+                        int mode, int g, uint16_t* What, int64_t ldo) {
+    int64_t G = K / g, GS = K / S;
+    float s_t = (mode == MODE_NVFP4) ? tensor_scale[0] : 1.f;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t e = n * K + k;
+            int sigma = sigma_bit(sigma_bits, n, GS, k / S);
+            float s = scale_value(scales, n * G + k / g, mode, s_t);
+            int c = (e & 1) ? (codes[e >> 1] >> 4) : (codes[e >> 1] & 0x0F);
+            What[n * ldo + k] = f32_to_bf16(bf16_to_f32(Tb[sigma * M + c]) * s);
+        }
+}
+
+double oracle_output_error_sel(const uint16_t* W, int64_t ldw, const uint8_t* codes, const void* scales,
+                               const float* tensor_scale, const uint16_t* Tb, const uint8_t* sigma_bits, int S,
+                               const float* I, int64_t N, int64_t K, int mode, int g) {
+    int64_t G = K / g, GS = K / S;
+    float s_t = (mode == MODE_NVFP4) ? tensor_scale[0] : 1.f;
+    double E = 0.0;
+    for (int64_t n = 0; n < N; ++n) {
+        double rowE = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t e = n * K + k;
+            int sigma = sigma_bit(sigma_bits, n, GS, k / S);
+            double s = (double)scale_value(scales, n * G + k / g, mode, s_t);
             int c = (e & 1) ? (codes[e >> 1] >> 4) : (codes[e >> 1] & 0x0F);
             double d = (double)bf16_to_f32(W[n * ldw + k]) - (double)bf16_to_f32(Tb[sigma * M + c]) * s;
             rowE += (double)I[k] * (d * d);
