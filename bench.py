@@ -176,6 +176,7 @@ def run_stack(args, which):
     if args.budget:                      # e.g. 3,10: the paper's default (n_outer, n_inner)
         rounds, n_inner = (int(v) for v in args.budget.split(","))
     g = 128 if mode == 0 else 16
+    sel = args.sel_group or None          # None: S = g, selection bit in the scale's sign
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     gen = torch.Generator(device=dev)
@@ -206,6 +207,7 @@ def run_stack(args, which):
                       ts=torch.ones(1, dtype=torch.float32, device=dev),
                       codes=torch.empty(N, K // 2, dtype=torch.uint8, device=dev),
                       err=torch.zeros(2, dtype=torch.float64, device=dev),
+                      bits=torch.empty(N, K // (8 * sel), dtype=torch.uint8, device=dev) if sel and sel != g else None,
                       ws=binding.alloc_workspace(mode, N, K, tokens, dev))
     Iv = {k: torch.empty(x.shape[1], dtype=torch.float32, device=dev) for k, x in X.items()}
     status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -216,9 +218,11 @@ def run_stack(args, which):
         for n, N, K, xin in lin:
             o = out[n]
             binding.fit_layer(Ws[n], mode, I=Iv[xin], n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE,
-                              T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
+                              T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status,
+                              sel_group=sel)
             binding.pack(Ws[n], mode, I=Iv[xin], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"],
-                         tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"])
+                         tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"], sel_group=sel,
+                         sigma_bits=o["bits"])
 
     for _ in range(2):
         decoder_layer()
@@ -238,7 +242,7 @@ def run_stack(args, which):
     line = {"metric": "aaac_stack_wall_s", "value": wall, "unit": "s", "n_gpus": 1, "higher_is_better": False,
             "dtype": "f32", "data": "synthetic (device-generated, one decoder layer's tensors reused for every layer)",
             "config": {"workload": f"{which}: {L} decoder layers x 7 linears (hidden {H}, kv {KV}, intermediate {FF}), "
-                                   f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'}, {tokens} tokens per input, quantile init, "
+                                   f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'} S{sel or g}, {tokens} tokens per input, quantile init, "
                                    f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds + pack",
                        "linears": 7 * L, "weights": wl * L, "rounds": rounds, "n_inner": n_inner},
             "gweights_per_s_per_round": wl * L * rounds * n_inner / wall / 1e9, "clocks": clocks}
@@ -258,6 +262,9 @@ def main():
                     help="cfg2 (default): the benchmark contract; stack8b / stack7b: wall time of a whole decoder stack")
     ap.add_argument("--budget", default="",
                     help="stack workloads only: n_outer,n_inner (default: the workload's rounds with n_inner = 1)")
+    ap.add_argument("--sel-group", type=int, default=0,
+                    help="stack workloads only: selection group size S (default: the scale group; 16 with stack8b "
+                         "is the paper's INT4 g128 S16 variant)")
     args = ap.parse_args()
     if args.workload != "cfg2":
         if int(os.environ.get("RANK", "0")) == 0:

@@ -158,6 +158,31 @@ int aaac_dequant(const uint8_t* codes, const void* scales, const float* tensor_s
                  void* What, int64_t ldo, void* stream);
 
 /*
+ * Selection group S smaller than the scale group g (Sec. 3.1, "granularity"; Algorithm 1
+ * line 20, "separately if S < g"): the same three calls with the selection group size given
+ * apart from the scale group.  Built for sel_group == group (then identical to the calls
+ * above; sigma_bits is ignored) and for the paper's INT4 variant group = 128, sel_group = 16;
+ * anything else returns AAAC_ERR_MODE.  With sel_group < group the selection costs 1/S bit per
+ * weight and lives in
+ *   sigma_bits  [N][K / (8 S)] bytes, row-major: selection group j of a row (columns
+ *               j S .. j S + S - 1) in bit j % 8 of the row's byte j / 8
+ * which aaac_pack_sel writes and aaac_dequant_sel reads, while the scales keep a clear sign
+ * bit.  aaac_fit_layer_sel's assignment step (Eq. 8) sums over selection groups of S weights.
+ */
+int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
+                       const float* I, const void* X, int64_t T, int64_t ldx,
+                       int n_outer, int n_inner, int init,
+                       float* T01, void* scales, float* tensor_scale, double* err_trace,
+                       uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+int aaac_pack_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
+                  const float* I, const float* T01_f32, uint16_t* T01_bf16,
+                  void* scales, const float* tensor_scale, uint8_t* codes, uint8_t* sigma_bits,
+                  double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, void* stream);
+int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* sigma_bits, const float* tensor_scale,
+                     const uint16_t* T01_bf16, int64_t N, int64_t K, int mode, int group, int sel_group,
+                     void* What, int64_t ldo, void* stream);
+
+/*
  * Whole path for one layer with HOST buffers: copies W and X to the device (into ws), runs
  * aaac_act_stats, aaac_fit_layer and aaac_pack, and copies tables, scales, tensor scale,
  * codes and errors back.  Host buffers should be page-locked for the copies to be

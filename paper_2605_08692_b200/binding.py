@@ -20,7 +20,7 @@ _lib = None
 
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
-           "aaac_timing_end"]
+           "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel"]
 
 
 class AaacError(RuntimeError):
@@ -48,11 +48,17 @@ def lib():
                                      C.c_size_t, vp]
         L.aaac_pack.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
         L.aaac_dequant.argtypes = [vp, vp, vp, vp, i64, i64, ci, ci, vp, i64, vp]
+        L.aaac_fit_layer_sel.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, vp, i64, i64, ci, ci, ci, vp, vp, vp, vp,
+                                         vp, vp, C.c_size_t, vp]
+        L.aaac_pack_sel.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                    C.c_size_t, vp]
+        L.aaac_dequant_sel.argtypes = [vp, vp, vp, vp, vp, i64, i64, ci, ci, ci, vp, i64, vp]
         L.aaac_quantize_layer_host.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                C.c_size_t, vp]
         L.aaac_timing_begin.argtypes = [ci]
         L.aaac_timing_end.argtypes = [vp, ci]
         for f in ("aaac_act_stats", "aaac_fit_layer", "aaac_pack", "aaac_dequant", "aaac_quantize_layer_host",
+                  "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel",
                   "aaac_timing_begin", "aaac_timing_end"):
             getattr(L, f).restype = C.c_int
         _lib = L
@@ -99,23 +105,40 @@ def act_stats_noalloc(X: torch.Tensor, I: torch.Tensor, accumulate: bool = False
 
 
 def fit_layer(W, mode, *, I=None, X=None, n_outer, init, T01, scales, tensor_scale, ws, err_trace=None,
-              dev_status=None, n_inner=1, group=None):
+              dev_status=None, n_inner=1, group=None, sel_group=None):
     N, K = W.shape
     T, ldx = (X.shape[0], X.stride(0)) if X is not None else (0, 0)
+    if sel_group is not None:
+        _check(lib().aaac_fit_layer_sel(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), sel_group, _ptr(I),
+                                        _ptr(X), T, ldx, n_outer, n_inner, init, _ptr(T01), _ptr(scales),
+                                        _ptr(tensor_scale), _ptr(err_trace), _ptr(dev_status), _ptr(ws), ws.numel(),
+                                        _stream()))
+        return
     _check(lib().aaac_fit_layer(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), _ptr(I), _ptr(X), T, ldx,
                                 n_outer, n_inner, init, _ptr(T01), _ptr(scales), _ptr(tensor_scale), _ptr(err_trace),
                                 _ptr(dev_status), _ptr(ws), ws.numel(), _stream()))
 
 
-def pack(W, mode, *, I, T01, T01_bf16, scales, tensor_scale, codes, ws, err_out=None, stats=None, group=None):
+def pack(W, mode, *, I, T01, T01_bf16, scales, tensor_scale, codes, ws, err_out=None, stats=None, group=None,
+         sel_group=None, sigma_bits=None):
     N, K = W.shape
+    if sel_group is not None:
+        _check(lib().aaac_pack_sel(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), sel_group, _ptr(I),
+                                   _ptr(T01), _ptr(T01_bf16), _ptr(scales), _ptr(tensor_scale), _ptr(codes),
+                                   _ptr(sigma_bits), _ptr(err_out), _ptr(stats), _ptr(ws), ws.numel(), _stream()))
+        return
     _check(lib().aaac_pack(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), _ptr(I), _ptr(T01),
                            _ptr(T01_bf16), _ptr(scales), _ptr(tensor_scale), _ptr(codes), _ptr(err_out), _ptr(stats),
                            _ptr(ws), ws.numel(), _stream()))
 
 
-def dequant(codes, scales, tensor_scale, T01_bf16, mode, What, group=None):
+def dequant(codes, scales, tensor_scale, T01_bf16, mode, What, group=None, sel_group=None, sigma_bits=None):
     N, K = What.shape
+    if sel_group is not None:
+        _check(lib().aaac_dequant_sel(_ptr(codes), _ptr(scales), _ptr(sigma_bits), _ptr(tensor_scale), _ptr(T01_bf16),
+                                      N, K, mode, group or group_of(mode), sel_group, _ptr(What), What.stride(0),
+                                      _stream()))
+        return
     _check(lib().aaac_dequant(_ptr(codes), _ptr(scales), _ptr(tensor_scale), _ptr(T01_bf16), N, K, mode,
                               group or group_of(mode), _ptr(What), What.stride(0), _stream()))
 
@@ -149,7 +172,8 @@ def timing_end(capacity: int):
 
 # ---- convenience for tests and the benchmark: allocate outputs, run the whole path ----
 
-def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trace=False, T01_init=None, n_inner=1):
+def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trace=False, T01_init=None, n_inner=1,
+                   sel_group=None):
     """Runs aaac_fit_layer then aaac_pack on device tensors and returns a dict of device tensors."""
     N, K = W.shape
     g = group_of(mode)
@@ -167,14 +191,17 @@ def quantize_layer(W, mode, *, I=None, X=None, n_outer, init, ws=None, want_trac
         I = torch.empty(K, dtype=torch.float32, device=dev)
         act_stats(X, I, ws, dev_status=status)
     fit_layer(W, mode, I=I, n_outer=n_outer, init=init, T01=T01, scales=scales, tensor_scale=ts, ws=ws,
-              err_trace=trace, dev_status=status, n_inner=n_inner)
+              err_trace=trace, dev_status=status, n_inner=n_inner, sel_group=sel_group)
     T01_fit = T01.clone()
     scales_pos = scales.clone()
     Tb = torch.empty(2, 16, dtype=torch.uint16, device=dev)
     codes = torch.empty(N, K // 2, dtype=torch.uint8, device=dev)
     err = torch.zeros(2, dtype=torch.float64, device=dev)
     stats = torch.zeros(4, dtype=torch.int64, device=dev)
+    sigma_bits = None
+    if sel_group is not None and sel_group != g:
+        sigma_bits = torch.empty(N, K // (8 * sel_group), dtype=torch.uint8, device=dev)
     pack(W, mode, I=I, T01=T01, T01_bf16=Tb, scales=scales, tensor_scale=ts, codes=codes, ws=ws, err_out=err,
-         stats=stats)
+         stats=stats, sel_group=sel_group, sigma_bits=sigma_bits)
     return dict(I=I, T01=T01_fit, T01_bf16=Tb, scales=scales, scales_pos=scales_pos, tensor_scale=ts, codes=codes,
-                err=err, stats=stats, trace=trace, status=status)
+                err=err, stats=stats, trace=trace, status=status, sigma_bits=sigma_bits)

@@ -46,6 +46,11 @@ Workspace carve(void* base, int mode, int64_t N, int64_t K) {
     return w;
 }
 
+// selection group sizes the kernels are built for: S = g, and S = 16 inside INT4's g = 128
+bool sel_ok(int mode, int group, int sel_group) {
+    return sel_group == group || (mode == AAAC_INT4 && group == 128 && sel_group == 16);
+}
+
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 int check_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group) {
@@ -119,8 +124,18 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
                    int n_outer, int n_inner, int init,
                    float* T01, void* scales, float* tensor_scale, double* err_trace,
                    uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+    return aaac_fit_layer_sel(W, N, K, ldw, mode, group, group, I, X, T, ldx, n_outer, n_inner, init, T01, scales,
+                              tensor_scale, err_trace, dev_status, ws, ws_bytes, stream);
+}
+
+int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
+                       const float* I, const void* X, int64_t T, int64_t ldx,
+                       int n_outer, int n_inner, int init,
+                       float* T01, void* scales, float* tensor_scale, double* err_trace,
+                       uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_layer(W, N, K, ldw, mode, group);
     if (rc) return rc;
+    if (!sel_ok(mode, group, sel_group)) return AAAC_ERR_MODE;
     if (!T01 || !scales || !tensor_scale) return AAAC_ERR_NULL;
     if (!I && !X) return AAAC_ERR_NULL;
     if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID && init != AAAC_INIT_USER) return AAAC_ERR_MODE;
@@ -156,7 +171,7 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
             }
         }
         if (e0) cudaEventRecord(e0, st);
-        if (launch_fit_rounds(Wp, N, K, ldw, mode, scales, I, n_outer, n_inner, err_trace, dev_status, w, st) != cudaSuccess)
+        if (launch_fit_rounds(Wp, N, K, ldw, mode, sel_group, scales, I, n_outer, n_inner, err_trace, dev_status, w, st) != cudaSuccess)
             return AAAC_ERR_CUDA;
         if (e1) cudaEventRecord(e1, st);
     }
@@ -167,8 +182,19 @@ int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int gr
               const float* I, const float* T01_f32, uint16_t* T01_bf16,
               void* scales, const float* tensor_scale, uint8_t* codes,
               double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, void* stream) {
+    return aaac_pack_sel(W, N, K, ldw, mode, group, group, I, T01_f32, T01_bf16, scales, tensor_scale, codes, nullptr,
+                         err_out, stats, ws, ws_bytes, stream);
+}
+
+int aaac_pack_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
+                  const float* I, const float* T01_f32, uint16_t* T01_bf16,
+                  void* scales, const float* tensor_scale, uint8_t* codes, uint8_t* sigma_bits,
+                  double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_layer(W, N, K, ldw, mode, group);
     if (rc) return rc;
+    if (!sel_ok(mode, group, sel_group)) return AAAC_ERR_MODE;
+    if (sel_group != group && !sigma_bits) return AAAC_ERR_NULL;
+    if (sel_group == group) sigma_bits = nullptr;
     if (!I || !T01_f32 || !T01_bf16 || !scales || !codes) return AAAC_ERR_NULL;
     if (mode == AAAC_NVFP4 && !tensor_scale) return AAAC_ERR_NULL;
     if (!aligned(I, 16) || !aligned(codes, 16) || !aligned(T01_bf16, 2)) return AAAC_ERR_ALIGN;
@@ -180,21 +206,30 @@ int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int gr
     if (cudaMemsetAsync(&w.ctrl->done, 0, sizeof(uint32_t), st) != cudaSuccess) return AAAC_ERR_CUDA;
     if (cudaMemsetAsync(w.ctrl->pack_err, 0, sizeof(double) * 2 + sizeof(unsigned long long) * 4, st) != cudaSuccess)
         return AAAC_ERR_CUDA;
-    return launch_pack(static_cast<const uint16_t*>(W), N, K, ldw, mode, I, T01_f32, T01_bf16, scales, tensor_scale,
-                       codes, err_out, reinterpret_cast<unsigned long long*>(stats), w, st) == cudaSuccess
+    return launch_pack(static_cast<const uint16_t*>(W), N, K, ldw, mode, sel_group, I, T01_f32, T01_bf16, scales,
+                       tensor_scale, codes, sigma_bits, err_out, reinterpret_cast<unsigned long long*>(stats), w, st) == cudaSuccess
                ? AAAC_OK : AAAC_ERR_CUDA;
 }
 
 int aaac_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale,
                  const uint16_t* T01_bf16, int64_t N, int64_t K, int mode, int group,
                  void* What, int64_t ldo, void* stream) {
+    return aaac_dequant_sel(codes, scales, nullptr, tensor_scale, T01_bf16, N, K, mode, group, group, What, ldo, stream);
+}
+
+int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* sigma_bits, const float* tensor_scale,
+                     const uint16_t* T01_bf16, int64_t N, int64_t K, int mode, int group, int sel_group,
+                     void* What, int64_t ldo, void* stream) {
     if (!codes || !scales || !T01_bf16 || !What) return AAAC_ERR_NULL;
     if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return AAAC_ERR_MODE;
     if (group != (mode == AAAC_INT4 ? 128 : 16)) return AAAC_ERR_MODE;
+    if (!sel_ok(mode, group, sel_group)) return AAAC_ERR_MODE;
+    if (sel_group != group && !sigma_bits) return AAAC_ERR_NULL;
+    if (sel_group == group) sigma_bits = nullptr;
     if (mode == AAAC_NVFP4 && !tensor_scale) return AAAC_ERR_NULL;
     if (N < 1 || K < 1 || K % group || K % 8 || ldo < K || ldo % 8) return AAAC_ERR_SHAPE;
     if (!aligned(codes, 4) || !aligned(What, 16)) return AAAC_ERR_ALIGN;
-    return launch_dequant(codes, scales, tensor_scale, T01_bf16, N, K, mode, static_cast<uint16_t*>(What), ldo,
+    return launch_dequant(codes, scales, sigma_bits, tensor_scale, T01_bf16, N, K, mode, static_cast<uint16_t*>(What), ldo,
                           static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
 

@@ -1,5 +1,6 @@
-// Dequantisation (Eq. 5): w^ = T_sigma[c] * s, with sigma the sign bit of the stored scale and s
-// its magnitude (times the tensor scale for NVFP4).  A pure stream: 0.5 byte of codes and a
+// Dequantisation (Eq. 5): w^ = T_sigma[c] * s, with sigma the sign bit of the stored scale (or,
+// when the selection group is 16 inside a scale group of 128, the group's bit of the separate
+// selection bytes) and s the scale's magnitude (times the tensor scale for NVFP4).  A pure stream: 0.5 byte of codes and a
 // scale per group in, 2 bytes out per weight.  Each thread expands one 32-bit word of codes
 // (8 weights) into one 128-bit store.
 #include "internal.cuh"
@@ -8,10 +9,10 @@ namespace aaac {
 
 namespace {
 
-template <int MODE>
+template <int MODE, bool SEP>
 __global__ void __launch_bounds__(256)
 dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scales,
-               const float* __restrict__ tensor_scale, const uint16_t* __restrict__ Tb,
+               const uint8_t* __restrict__ sigma_bits, const float* __restrict__ tensor_scale, const uint16_t* __restrict__ Tb,
                int64_t N, int64_t K, uint16_t* __restrict__ What, int64_t ldo) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     __shared__ float T[2 * kM];
@@ -36,6 +37,7 @@ dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             sigma = b >> 7;
             s = slut[b & 0x7Fu];
         }
+        if (SEP) sigma = (sigma_bits[row * (K >> 7) + (col >> 7)] >> ((col >> 4) & 7)) & 1u;
         const float* Ts = T + sigma * kM;
         uint32_t o[4];
 #pragma unroll
@@ -50,16 +52,19 @@ dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
 
 }  // namespace
 
-cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale, const uint16_t* Tb,
-                           int64_t N, int64_t K, int mode, uint16_t* What, int64_t ldo, cudaStream_t st) {
+cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const uint8_t* sigma_bits,
+                           const float* tensor_scale, const uint16_t* Tb, int64_t N, int64_t K, int mode,
+                           uint16_t* What, int64_t ldo, cudaStream_t st) {
     const int64_t total = N * (K / 8);
     int64_t blocks = (total + 255) / 256;
     const int64_t cap = (int64_t)sm_count() * 16;
     if (blocks > cap) blocks = cap;
-    if (mode == AAAC_INT4)
-        dequant_kernel<AAAC_INT4><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, tensor_scale, Tb, N, K, What, ldo);
+    if (mode == AAAC_INT4 && sigma_bits)
+        dequant_kernel<AAAC_INT4, true><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, sigma_bits, tensor_scale, Tb, N, K, What, ldo);
+    else if (mode == AAAC_INT4)
+        dequant_kernel<AAAC_INT4, false><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, nullptr, tensor_scale, Tb, N, K, What, ldo);
     else
-        dequant_kernel<AAAC_NVFP4><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, tensor_scale, Tb, N, K, What, ldo);
+        dequant_kernel<AAAC_NVFP4, false><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, nullptr, tensor_scale, Tb, N, K, What, ldo);
     return cudaGetLastError();
 }
 

@@ -135,11 +135,13 @@ __device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
 // single pass followed by one kInner launch of n_inner - 1 passes.
 enum PassKind { kRounds = 0, kAssignKeep = 1, kInner = 2 };
 
-template <int MODE, int NW, int REP, int KIND>
+// SEL is the selection group size S (Sec. 3.1): the weights that share one codebook choice; the
+// scale group g is fixed by the format.
+template <int MODE, int SEL, int NW, int REP, int KIND>
 __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
     constexpr int NB = AAAC_FIT_BINS;
-    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
-    constexpr int LPG = G / 8;
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
+    constexpr int LPG = SEL / 8;                         // lanes per selection group
     constexpr int R = kRowsPerWarp;
     constexpr int kRowsPerItem = R * NW;
     constexpr int NT = NW * 32;
@@ -521,10 +523,10 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
     if (threadIdx.x < 2 * kM) T01[threadIdx.x] = (float)ctrl->T[threadIdx.x];
 }
 
-template <int MODE, int NW, int REP, int KIND>
+template <int MODE, int SEL, int NW, int REP, int KIND>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
-    auto kern = fit_rounds_kernel<MODE, NW, REP, KIND>;
+    auto kern = fit_rounds_kernel<MODE, SEL, NW, REP, KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&p};
@@ -534,7 +536,7 @@ cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
 
 }  // namespace
 
-cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
+cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
                               const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st) {
     if (n_outer <= 0) return cudaSuccess;
@@ -558,8 +560,9 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
     auto launch = [&](auto kind) {
         constexpr int KIND = decltype(kind)::value;
-        if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, NW, REP, KIND>(p, (unsigned)grid, st);
-        return launch_variant<AAAC_NVFP4, NW, REP, KIND>(p, (unsigned)grid, st);
+        if (mode == AAAC_INT4 && sel_group == 16) return launch_variant<AAAC_INT4, 16, NW, REP, KIND>(p, (unsigned)grid, st);
+        if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, 128, NW, REP, KIND>(p, (unsigned)grid, st);
+        return launch_variant<AAAC_NVFP4, 16, NW, REP, KIND>(p, (unsigned)grid, st);
     };
     if (n_inner == 1) return launch(std::integral_constant<int, kRounds>{});
     for (int outer = 0; outer < n_outer; ++outer) {

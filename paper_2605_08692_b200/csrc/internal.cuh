@@ -99,16 +99,18 @@ cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, 
                           float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
                         const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st);
-cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const void* scales,
+cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
                               const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st);
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st);
-cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,
+// sigma_bits: null when the selection group is the scale group (sigma in the scale's sign bit)
+cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const float* I,
                         const float* T01_f32, uint16_t* T01_bf16, void* scales, const float* tensor_scale,
-                        uint8_t* codes, double* err_out, unsigned long long* stats, const Workspace& ws,
-                        cudaStream_t st);
-cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale, const uint16_t* Tb,
-                           int64_t N, int64_t K, int mode, uint16_t* What, int64_t ldo, cudaStream_t st);
+                        uint8_t* codes, uint8_t* sigma_bits, double* err_out, unsigned long long* stats,
+                        const Workspace& ws, cudaStream_t st);
+cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const uint8_t* sigma_bits,
+                           const float* tensor_scale, const uint16_t* Tb, int64_t N, int64_t K, int mode,
+                           uint16_t* What, int64_t ldo, cudaStream_t st);
 
 int sm_count();
 

@@ -40,6 +40,7 @@ struct PackParams {
     const float* T01_f32;
     uint16_t* T01_bf16;
     uint8_t* codes;
+    uint8_t* sigma_bits;          // [N][K / 128] when the selection group is 16 inside a scale group of 128; else null
     int items, per_block, nrb;
 };
 
@@ -56,10 +57,11 @@ __device__ __noinline__ int count_idx_ties(const FitTables* S, Row8 r, int sg) {
     return n;
 }
 
-template <int MODE, int NW, int REP>
+template <int MODE, int SEL, int NW, int REP>
 __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
-    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
-    constexpr int LPG = G / 8;
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
+    constexpr int LPG = SEL / 8;                         // lanes per selection group
+    static_assert(SEL == G || SEL == 16, "separate selection bits are laid out for groups of 16");
     constexpr int R = kRowsPerWarp;
     constexpr int kRowsPerItem = R * NW;
     constexpr int kLut1Bytes = REP * kNBins * 8;
@@ -227,6 +229,17 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
                     if (col_ok && (lane % LPG) == 0) { ++n_exact; n_sig_tie += ex.tie; }
                 }
             }
+            if (SEL != G) {
+                // selection bits apart (Algorithm 1 line 20, S < g): group j of the row in bit j % 8 of
+                // byte j / 8; a row's 256-column slab holds 16 groups, led by the even lanes
+                uint32_t b = __ballot_sync(0xFFFFFFFFu, sg) & 0x55555555u;
+                b = (b | (b >> 1)) & 0x33333333u;
+                b = (b | (b >> 2)) & 0x0F0F0F0Fu;
+                b = (b | (b >> 4)) & 0x00FF00FFu;
+                b = (b | (b >> 8)) & 0x0000FFFFu;
+                if (col_ok && (lane & 15) == 0)
+                    p.sigma_bits[(size_t)row * (size_t)(K >> 7) + (uint32_t)col0 / 128u] = (uint8_t)(b >> (lane >> 1));
+            }
             if (!col_ok) continue;
             if ((lane % LPG) == 0) Eacc += emin;
             // codes (Eq. 6) and the error in weight units
@@ -249,7 +262,7 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
                 n_idx_tie += count_idx_ties(&S, r, (int)sg);
             }
             *reinterpret_cast<uint32_t*>(p.codes + (((size_t)row * (size_t)K + col0) >> 1)) = word;
-            if ((lane % LPG) == 0) {
+            if (SEL == G && (lane % LPG) == 0) {
                 const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
                 if (MODE == AAAC_NVFP4)
                     reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
@@ -304,10 +317,10 @@ __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long lo
     }
 }
 
-template <int MODE>
+template <int MODE, int SEL>
 cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kJSlots * kSlotBytes;
-    auto kern = pack_kernel<MODE, kPackWarps, kPackRep>;
+    auto kern = pack_kernel<MODE, SEL, kPackWarps, kPackRep>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, kPackWarps * 32, smem, st>>>(p);
@@ -316,14 +329,15 @@ cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t
 
 }  // namespace
 
-cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, const float* I,
+cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const float* I,
                         const float* T01_f32, uint16_t* T01_bf16, void* scales, const float* tensor_scale,
-                        uint8_t* codes, double* err_out, unsigned long long* stats, const Workspace& ws,
-                        cudaStream_t st) {
+                        uint8_t* codes, uint8_t* sigma_bits, double* err_out, unsigned long long* stats,
+                        const Workspace& ws, cudaStream_t st) {
     PackParams p{};
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
     p.scales = scales; p.I = I; p.tensor_scale = tensor_scale;
     p.ctrl = ws.ctrl; p.part = ws.part; p.T01_f32 = T01_f32; p.T01_bf16 = T01_bf16; p.codes = codes;
+    p.sigma_bits = sigma_bits;
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * kPackWarps;
     const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
@@ -334,8 +348,10 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     const int64_t per_block = (items + grid - 1) / grid;
     grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
-    cudaError_t e = mode == AAAC_INT4 ? launch_pack_variant<AAAC_INT4>(p, (unsigned)grid, st)
-                                      : launch_pack_variant<AAAC_NVFP4>(p, (unsigned)grid, st);
+    cudaError_t e;
+    if (mode == AAAC_INT4 && sel_group == 16) e = launch_pack_variant<AAAC_INT4, 16>(p, (unsigned)grid, st);
+    else if (mode == AAAC_INT4) e = launch_pack_variant<AAAC_INT4, 128>(p, (unsigned)grid, st);
+    else e = launch_pack_variant<AAAC_NVFP4, 16>(p, (unsigned)grid, st);
     if (e != cudaSuccess) return e;
     export_pack_kernel<<<1, 32, 0, st>>>(ws.ctrl, err_out, stats);
     return cudaGetLastError();

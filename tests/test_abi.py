@@ -74,6 +74,14 @@ def test_argument_validation_happens_on_the_host(L):
     assert fit(I=None) == 1
     assert fit(wsb=C.c_size_t(1024)) == 5
     assert fit(ws=P((1 << 20) + 64)) == 4
+    # selection group apart from the scale group: S = g, or S = 16 inside INT4's g = 128
+    fits = lambda mode, group, sel: L.aaac_fit_layer_sel(ok, 64, 256, 256, mode, group, sel, ok, None, 0, 0, 2, 1, 1, ok,
+                                                         ok, ok, None, None, ok, C.c_size_t(16), None)
+    assert fits(0, 128, 16) == 5 and fits(0, 128, 128) == 5 and fits(1, 16, 16) == 5     # pass the checks up to the workspace size
+    assert fits(0, 128, 32) == 2 and fits(1, 16, 8) == 2 and fits(1, 16, 128) == 2
+    assert L.aaac_pack_sel(ok, 64, 256, 256, 0, 128, 16, ok, ok, ok, ok, ok, ok, None, None, None, ok, big, None) == 1
+    assert L.aaac_dequant_sel(ok, ok, None, ok, ok, 64, 256, 0, 128, 16, ok, 256, None) == 1
+    assert L.aaac_dequant_sel(ok, ok, ok, ok, ok, 64, 256, 0, 128, 64, ok, 256, None) == 2
     # aaac_pack / aaac_dequant
     assert L.aaac_pack(ok, 64, 256, 256, 0, 128, None, ok, ok, ok, ok, ok, None, None, ok, big, None) == 1
     assert L.aaac_pack(ok, 64, 256, 256, 1, 16, ok, ok, ok, ok, None, ok, None, None, ok, big, None) == 1
