@@ -1,9 +1,10 @@
 // The fit rounds (Algorithm 1 lines 6-16).  With n_inner = 1 a round is the assignment step
 // (Eq. 8) and the activation-weighted centroid update (Eq. 11) in a single pass over W, and all
 // rounds of a layer run in ONE persistent kernel (one block per SM, cooperative launch): after
-// its pass every block publishes a partial, the blocks meet at a grid-wide barrier, and every
-// block adds all partials in the same fixed order, so each holds the same new tables without a
-// second barrier or a relaunch.  The barrier wait is bounded: if it runs out, the kernel sets
+// its pass every block adds its sums, as 96-bit fixed-point integers, into 65 global accumulators,
+// the blocks meet at a grid-wide barrier, and every block reads the totals, so each holds the
+// same new tables without a second barrier or a relaunch (integer addition does not depend on
+// the order in which the blocks arrive, so the result is bitwise reproducible).  The barrier wait is bounded: if it runs out, the kernel sets
 // AAAC_DEV_TIMEOUT in the device status word and returns.
 // With n_inner > 1 the assignment pass (which is also the first inner iteration) stores the
 // selection bits, one word per row and 256-column slab, and the remaining n_inner - 1 inner
@@ -47,9 +48,9 @@
 // (c) Centroid sums, centred.  Lane-private shared-memory bins [sigma][entry] hold
 //     (sum I (x - c), sum I) with c the constant of (b) for the entry the weight is assigned to,
 //     so the new entry is c + sum I (x - c) / sum I.  The residual sums are small and of mixed
-//     sign, which keeps the FP32 accumulation error some 20 times below that of sum I x.  No
-//     atomics, fixed order.  One partial per block and round; after the barrier the partials are
-//     added in a fixed order, the centroids formed (entries of empty cells keep their value) and
+//     sign, which keeps the FP32 accumulation error some 20 times below that of sum I x.  Within
+//     a block: no atomics, fixed order.  Across blocks: integer atomics (see above).  After the
+//     barrier the centroids are formed (entries of empty cells keep their value) and
 //     sorted; block 0 stores the Eq. 8 objective of the round (sum over groups of the smaller
 //     error) and, after the last round, the tables.
 //
@@ -77,7 +78,7 @@ struct FitParams {
     const float* rinv;            // INT4 reciprocal scales
     const float* I;
     Ctrl* ctrl;
-    double* part;                 // [2][kMaxBlocks][kPartStride]: partials of even / odd rounds
+    unsigned long long* acc;      // [3][kUsed][3]: fixed-point sums over the blocks, one buffer per pass in rotation
     double* err_trace;            // [n_rounds] or null
     uint32_t* dev_status;         // or null
     uint32_t* sigw;               // [N][slabs]: selection bits of a row's 256-column slab, bit = lane (n_inner > 1)
@@ -98,7 +99,8 @@ __device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
     lo = __fadd_rn(lo, err);
 }
 
-constexpr int kMaxFitBlocks = 192;                    // grid limit: the partials of all blocks are staged in shared memory
+constexpr int kMaxFitBlocks = 1024;                   // grid limit: block sums are added as 32-bit limbs in 64-bit words
+constexpr int kLimbs = 3;                             // a sum is a 96-bit two's-complement fixed-point number
 constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
 
 // Grid-wide barrier of a cooperative launch: block arrivals are counted in ctrl->bar, which only
@@ -176,6 +178,29 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         S.rlut[c] = c ? __frcp_rn(sv) : 0.f;
     }
     __syncthreads();
+
+    // Fixed-point scale of the sums over the blocks.  Every sum of a pass is bounded by
+    // B = 256 N K max_k I_k (|w~ - c| < 16), so with 2^e > B the value v 2^(94 - e) fits 96 bits; what
+    // is dropped lies 2^-86 below B.  Integer addition is order-independent, so the totals do not
+    // depend on the order in which the blocks arrive (max is order-independent too).
+    {
+        float mx = 0.f;
+        for (int k = tid; k < K; k += NT) mx = fmaxf(mx, fabsf(__ldg(p.I + k)));
+#pragma unroll
+        for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        float* red = reinterpret_cast<float*>(dyn);
+        if (lane == 0) red[warp] = mx;
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < NW; ++w) mx = fmaxf(mx, red[w]);
+            const double B = 256.0 * (double)N * (double)K * (double)mx;
+            int e = 0;
+            if (B > 0.0 && B < 1e300) e = ilogb(B) + 1;
+            S.fix_scale = scalbn(1.0, 94 - e);
+            S.fix_unscale = scalbn(1.0, e - 94);
+        }
+        __syncthreads();
+    }
 
     // bin arithmetic: the masked mantissa of fl32(kBinsPerUnit x + kMagic) is bin * (REP * 8)
     constexpr float kBinsPerUnit = (float)(NB / 16);
@@ -448,52 +473,40 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     for (int s = 16; s; s >>= 1) Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, s);
     if (lane == 0) wsum[warp * kPartStride + 2 * kCells] = Eacc;
     __syncthreads();
-    // a partial is stored as an FP32 pair (hi, lo) of its double value: exact to 2^-48
-    float2* part = reinterpret_cast<float2*>(p.part + (size_t)(round & 1) * kMaxBlocks * kPartStride);
+    // this block's sums go into the pass's buffer as three 32-bit limbs of a 96-bit fixed-point number
+    const unsigned pass_no = p.bar_base + (unsigned)round;
+    unsigned long long* acc = p.acc + (size_t)(pass_no % 3u) * (kUsed * kLimbs);
     if (tid < kUsed) {
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < NW; ++w) s += wsum[w * kPartStride + tid];
-        const float hi = (float)s;
-        part[(size_t)blockIdx.x * kPartStride + tid] = make_float2(hi, (float)(s - (double)hi));
+        const double sd = s * S.fix_scale;
+        const double t2 = floor(sd * 0x1p-64);
+        const double r = sd - t2 * 0x1p64;                 // exact, in [0, 2^64)
+        const double t1 = floor(r * 0x1p-32);
+        const double t0 = floor(r - t1 * 0x1p32);
+        atomicAdd(acc + tid * kLimbs + 0, (unsigned long long)t0);
+        atomicAdd(acc + tid * kLimbs + 1, (unsigned long long)t1);
+        atomicAdd(acc + tid * kLimbs + 2, (unsigned long long)(long long)t2);
     }
+    // block 0 clears the next pass's buffer: every block has finished reading it (it was the buffer
+    // of two passes ago) before block 0 could leave the previous barrier
+    if (blockIdx.x == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs)
+        p.acc[(size_t)((pass_no + 1u) % 3u) * (kUsed * kLimbs) + (tid - 256)] = 0ull;
 
-    // ---- all blocks meet; then each adds the partials of all blocks in the same fixed order
-    //      (kStrands interleaved strands per value, each in block order, then the strands) ----
-    if (!grid_barrier(S, p.ctrl, (p.bar_base + (unsigned)round + 1u) * gridDim.x)) {
+    // ---- all blocks meet; then each reads the totals ----
+    if (!grid_barrier(S, p.ctrl, (pass_no + 1u) * gridDim.x)) {
         if (blockIdx.x == 0 && tid == 0 && p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
         return;
     }
-    {
-        // stage every block's partial in shared memory (the bins' space; all loads independent),
-        // then add them per value in kStrands interleaved strands, each in block order
-        static_assert((size_t)NW * kBinBytes >= (size_t)kMaxFitBlocks * kUsed * sizeof(float2), "staging space");
-        float2* stage = reinterpret_cast<float2*>(dyn + kLut1Bytes + kLut2Bytes);      // [grid][kUsed]
-        const int total = (int)gridDim.x * kUsed;
-#pragma unroll 8
-        for (int i = tid; i < total; i += NT) {
-            const int b = i / kUsed;
-            stage[i] = __ldcg(part + (size_t)b * kPartStride + (i - b * kUsed));
-        }
-        __syncthreads();
-        constexpr int kStrands = NT / kUsed;
-        const int strand = tid / kUsed, val = tid - strand * kUsed;
-        if (strand < kStrands) {
-            float hi = 0.f, lo = 0.f;
-            for (int b = strand; b < (int)gridDim.x; b += kStrands) {
-                const float2 v = stage[b * kUsed + val];
-                two_sum(hi, lo, v.x);
-                lo = __fadd_rn(lo, v.y);
-            }
-            wsum[strand * kPartStride + val] = (double)hi + (double)lo;
-        }
-        __syncthreads();
-        if (tid < kUsed) {
-            double t = 0.0;
-#pragma unroll
-            for (int k = 0; k < kStrands; ++k) t += wsum[k * kPartStride + tid];
-            S.tot[tid] = t;
-        }
+    if (tid < kUsed) {
+        const unsigned long long l0 = __ldcg(acc + tid * kLimbs + 0), l1 = __ldcg(acc + tid * kLimbs + 1);
+        const long long l2 = (long long)__ldcg(acc + tid * kLimbs + 2);
+        __int128 v = ((__int128)l2 << 64) + ((__int128)l1 << 32) + (__int128)l0;
+        const bool neg = v < 0;
+        if (neg) v = -v;
+        const double mag = (double)(unsigned long long)(v >> 64) * 0x1p64 + (double)(unsigned long long)v;
+        S.tot[tid] = (neg ? -mag : mag) * S.fix_unscale;
     }
     __syncthreads();
     if (tid < 2 * kM) {
@@ -544,7 +557,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     FitParams p{};
     p.W = W; p.N = N; p.K = K; p.ldw = ldw;
     p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
-    p.ctrl = ws.ctrl; p.part = ws.part; p.err_trace = err_trace; p.dev_status = dev_status;
+    p.ctrl = ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(ws.part); p.err_trace = err_trace; p.dev_status = dev_status;
     p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
     p.sigw = ws.qlist;            // the quantile selection's list is free once the start tables exist
     const int64_t slabs = (K + 255) / 256;
@@ -564,6 +577,9 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
         if (mode == AAAC_INT4) return launch_variant<AAAC_INT4, 128, NW, REP, KIND>(p, (unsigned)grid, st);
         return launch_variant<AAAC_NVFP4, 16, NW, REP, KIND>(p, (unsigned)grid, st);
     };
+    // the three rotating sum buffers start at zero
+    cudaError_t em = cudaMemsetAsync(p.acc, 0, sizeof(unsigned long long) * 3 * kUsed * kLimbs, st);
+    if (em != cudaSuccess) return em;
     if (n_inner == 1) return launch(std::integral_constant<int, kRounds>{});
     for (int outer = 0; outer < n_outer; ++outer) {
         p.n_rounds = 1; p.trace_base = outer;

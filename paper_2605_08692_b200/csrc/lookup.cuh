@@ -86,6 +86,7 @@ struct FitTables {
     float tmax283;                // 2.83 * 17 * max |entry|, rounded up
     int is_last;
     double tot[kPartStride];
+    double fix_scale, fix_unscale;   // fit rounds: fixed-point scale of the sums over the blocks and its inverse
 };
 
 // Builds every lookup table of the round from the current tables in S.Td.
