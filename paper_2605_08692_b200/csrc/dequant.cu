@@ -21,32 +21,52 @@ dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
     if (MODE == AAAC_NVFP4 && threadIdx.x >= 128)
         slut[threadIdx.x - 128] = __fmul_rn(e4m3_value(threadIdx.x - 128), tensor_scale[0]);
     __syncthreads();
-    const int64_t per_row = K / 8, total = N * per_row, Gr = K / G;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = i / per_row, col = (i % per_row) * 8;
-        const uint32_t word = __ldcs(reinterpret_cast<const uint32_t*>(codes + ((row * K + col) >> 1)));
-        const int64_t gi = row * Gr + col / G;
-        uint32_t sigma;
-        float s;
-        if (MODE == AAAC_INT4) {
-            const uint32_t b = reinterpret_cast<const uint16_t*>(scales)[gi];
-            sigma = b >> 15;
-            s = __uint_as_float((b & 0x7FFFu) << 16);
-        } else {
-            const uint32_t b = reinterpret_cast<const uint8_t*>(scales)[gi];
-            sigma = b >> 7;
-            s = slut[b & 0x7Fu];
-        }
-        if (SEP) sigma = (sigma_bits[row * (K >> 7) + (col >> 7)] >> ((col >> 4) & 7)) & 1u;
-        const float* Ts = T + sigma * kM;
-        uint32_t o[4];
+    const int64_t per_row = K / 8, Gr = K / G;
+    // two independent items in flight per thread, no division per item
+    SlabWalk it((int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x, per_row);
+    while (it.row < N) {
+        int64_t rows[2], cols[2];
+        uint32_t words[2], sb[2], sgb[2];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t lo = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j)) & 15u], s));
-            const uint32_t hi = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j + 4)) & 15u], s));
-            o[j] = lo | (hi << 16);
+        for (int u = 0; u < 2; ++u) {
+            rows[u] = it.row;
+            cols[u] = (int64_t)it.slab * 8;
+            words[u] = 0u; sb[u] = 0u; sgb[u] = 0u;
+            if (it.row < N) {
+                const int64_t row = rows[u], col = cols[u];
+                words[u] = __ldcs(reinterpret_cast<const uint32_t*>(codes + ((row * K + col) >> 1)));
+                const int64_t gi = row * Gr + col / G;
+                sb[u] = MODE == AAAC_INT4 ? (uint32_t)reinterpret_cast<const uint16_t*>(scales)[gi]
+                                          : (uint32_t)reinterpret_cast<const uint8_t*>(scales)[gi];
+                if (SEP) sgb[u] = sigma_bits[row * (K >> 7) + (col >> 7)];
+            }
+            it.next();
         }
-        __stcs(reinterpret_cast<uint4*>(What + row * ldo + col), make_uint4(o[0], o[1], o[2], o[3]));
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (rows[u] >= N) break;
+            const int64_t row = rows[u], col = cols[u];
+            const uint32_t word = words[u], b = sb[u];
+            uint32_t sigma;
+            float s;
+            if (MODE == AAAC_INT4) {
+                sigma = b >> 15;
+                s = __uint_as_float((b & 0x7FFFu) << 16);
+            } else {
+                sigma = b >> 7;
+                s = slut[b & 0x7Fu];
+            }
+            if (SEP) sigma = (sgb[u] >> ((col >> 4) & 7)) & 1u;
+            const float* Ts = T + sigma * kM;
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t lo = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j)) & 15u], s));
+                const uint32_t hi = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j + 4)) & 15u], s));
+                o[j] = lo | (hi << 16);
+            }
+            __stcs(reinterpret_cast<uint4*>(What + row * ldo + col), make_uint4(o[0], o[1], o[2], o[3]));
+        }
     }
 }
 

@@ -11,7 +11,8 @@
 //      into a slotted bin to that slot's list -- the lists' sizes are known from step 1.  A block
 //      stages its candidates in shared memory and reserves list space once per slot, so the
 //      global counters see one atomic per block and slot instead of one per candidate;
-//   4. one block per slot selects the requested ranks of its list by an 8-bit radix select;
+//   4. one block per slot selects the requested ranks of its list by an 8-bit radix select (the
+//      list is read once into registers when it is short enough, else streamed per pass);
 //   5. the table entries are interpolated in double and rounded to FP32.
 // Integer atomics only, so the result does not depend on scheduling.
 //
@@ -47,7 +48,7 @@ __device__ __forceinline__ float group_rinv(const void* scales, int64_t gi, floa
 }
 
 // Step 1: histogram of every w~ (shared-memory counters per block, merged with integer atomics).
-// A warp takes two 256-column pieces per iteration so that two loads are in flight.
+// A warp takes four 256-column pieces per iteration so that four loads are in flight.
 template <int MODE>
 __global__ void __launch_bounds__(256)
 quantile_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
@@ -58,27 +59,28 @@ quantile_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64
     for (int i = threadIdx.x; i < kQBins; i += blockDim.x) sm[i] = 0;
     __syncthreads();
     const float s_t = ctrl->s_t;
-    const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
+    const int64_t slabs = (K + 255) / 256, Gr = K / G;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    for (int64_t it = warp0; it < items; it += 2 * nwarps) {
-        uint4 v[2];
-        float r[2];
-        bool ok[2];
+    SlabWalk it(warp0, nwarps, slabs);
+    while (it.row < N) {
+        uint4 v[4];
+        float r[4];
+        bool ok[4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int64_t i2 = it + h * nwarps;
-            const int64_t row = i2 / slabs, col = (i2 % slabs) * 256 + lane * 8;
-            ok[h] = i2 < items && col < K;
+        for (int h = 0; h < 4; ++h) {
+            const int64_t row = it.row, col = (int64_t)it.slab * 256 + lane * 8;
+            ok[h] = row < N && col < K;
             v[h] = make_uint4(0, 0, 0, 0);
             r[h] = 0.f;
             if (ok[h]) {
                 v[h] = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
                 r[h] = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
             }
+            it.next();
         }
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < 4; ++h) {
             if (!ok[h]) continue;
             const uint32_t w[4] = {v[h].x, v[h].y, v[h].z, v[h].w};
 #pragma unroll
@@ -279,6 +281,25 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     const unsigned long long n = ctrl->slot_off[slot + 1] - ctrl->slot_off[slot];
     const unsigned long long n_up = (n + blockDim.x - 1) / blockDim.x * blockDim.x;
     const int lane = threadIdx.x & 31;
+    // A list of up to kKeep keys per thread is read once and kept in registers for every pass of
+    // every request of the slot; longer lists are streamed from memory in each pass.
+    constexpr int kKeep = 24;
+    const bool kept = n <= (unsigned long long)kKeep * blockDim.x;
+    uint32_t kc[kKeep];
+#pragma unroll
+    for (int u = 0; u < kKeep; ++u) {
+        const unsigned long long i = threadIdx.x + (unsigned long long)u * blockDim.x;
+        kc[u] = (kept && i < n) ? keys[i] : 0u;
+    }
+    // one key's vote for its digit: equal digits within a warp are counted once
+    auto vote = [&](uint32_t k, bool sel, int shift) {
+        const unsigned act = __ballot_sync(0xFFFFFFFFu, sel);
+        if (sel) {
+            const uint32_t d = (k >> shift) & 0xFFu;
+            const unsigned peers = __match_any_sync(act, d);
+            if (lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+        }
+    };
     __syncthreads();
     for (int q = 0; q < kQReq; ++q) {
         if (req_slot[q] != slot) continue;                 // uniform across the block
@@ -288,6 +309,14 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
             if (threadIdx.x < 256) hist[threadIdx.x] = 0;
             __syncthreads();
             const uint32_t prefix = sh_prefix, mask = sh_mask;
+            if (kept) {
+#pragma unroll
+                for (int u = 0; u < kKeep; ++u) {
+                    if ((unsigned long long)u * blockDim.x >= n_up) break;      // uniform over the block
+                    const unsigned long long i = threadIdx.x + (unsigned long long)u * blockDim.x;
+                    vote(kc[u], i < n && (kc[u] & mask) == prefix, shift);
+                }
+            } else
             for (unsigned long long i0 = threadIdx.x; i0 < n_up; i0 += 4ull * blockDim.x) {
                 uint32_t kk[4];
 #pragma unroll
@@ -299,14 +328,7 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
                 for (int u = 0; u < 4; ++u) {
                     const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
                     if (i >= n_up) break;                  // uniform over the block
-                    const uint32_t k = kk[u];
-                    const bool sel = i < n && (k & mask) == prefix;
-                    const unsigned act = __ballot_sync(0xFFFFFFFFu, sel);
-                    if (sel) {
-                        const uint32_t d = (k >> shift) & 0xFFu;
-                        const unsigned peers = __match_any_sync(act, d);
-                        if (lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
-                    }
+                    vote(kk[u], i < n && (kk[u] & mask) == prefix, shift);
                 }
             }
             __syncthreads();

@@ -89,6 +89,20 @@ __device__ __forceinline__ uint32_t e4m3_encode(float x) {
     return u > 0x7Eu ? 0x7Eu : u;
 }
 
+// Walks the items first, first + stride, first + 2 stride, ... of an N x slabs grid (row-major)
+// without a division per step; row runs past N when the walk is over.
+struct SlabWalk {
+    int row, slab, drow, dslab, slabs;
+    __device__ SlabWalk(int64_t first, int64_t stride, int64_t slabs_)
+        : row((int)(first / slabs_)), slab((int)(first % slabs_)), drow((int)(stride / slabs_)),
+          dslab((int)(stride % slabs_)), slabs((int)slabs_) {}
+    __device__ void next() {
+        row += drow;
+        slab += dslab;
+        if (slab >= slabs) { slab -= slabs; ++row; }
+    }
+};
+
 // largest float <= d
 __device__ __forceinline__ float f32_round_down(double d) { return __double2float_rd(d); }
 

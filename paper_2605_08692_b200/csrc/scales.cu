@@ -30,13 +30,23 @@ __device__ __forceinline__ uint32_t absmax16(uint4 v) {
 __global__ void __launch_bounds__(256)
 absmax_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, Ctrl* ctrl) {
     const int lane = threadIdx.x & 31;
-    const int64_t slabs = (K + 255) / 256, items = N * slabs;
+    const int64_t slabs = (K + 255) / 256;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     uint32_t m = 0;
-    for (int64_t it = warp0; it < items; it += nwarps) {
-        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
-        if (col < K) m = max(m, absmax16(__ldg(reinterpret_cast<const uint4*>(W + row * ldw + col))));
+    // four independent loads in flight per thread
+    SlabWalk it(warp0, nwarps, slabs);
+    while (it.row < N) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            v[u] = make_uint4(0, 0, 0, 0);
+            const int64_t col = (int64_t)it.slab * 256 + lane * 8;
+            if (it.row < N && col < K) v[u] = __ldg(reinterpret_cast<const uint4*>(W + (int64_t)it.row * ldw + col));
+            it.next();
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) m = max(m, absmax16(v[u]));
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -53,7 +63,7 @@ scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;                         // lanes per group
     const int lane = threadIdx.x & 31;
-    const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
+    const int64_t slabs = (K + 255) / 256, Gr = K / G;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
 
@@ -69,10 +79,24 @@ scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
         if (tensor_scale) tensor_scale[0] = s_t;
     }
     bool bad = false;
-    for (int64_t it = warp0; it < items; it += nwarps) {
-        const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
-        uint32_t m = 0;
-        if (col < K) m = absmax16(__ldg(reinterpret_cast<const uint4*>(W + row * ldw + col)));
+    SlabWalk it(warp0, nwarps, slabs);
+    while (it.row < N) {
+      // four independent loads in flight per thread (the row of an item is the same in every lane)
+      uint4 v[4];
+      int rows[4], cols[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+          v[u] = make_uint4(0, 0, 0, 0);
+          rows[u] = it.row;
+          cols[u] = it.slab * 256 + lane * 8;
+          if (it.row < N && cols[u] < K) v[u] = __ldg(reinterpret_cast<const uint4*>(W + (int64_t)it.row * ldw + cols[u]));
+          it.next();
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (rows[u] >= N) break;                       // uniform over the warp
+        const int64_t row = rows[u], col = cols[u];
+        uint32_t m = absmax16(v[u]);
 #pragma unroll
         for (int o = LPG / 2; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
         if (col < K && (lane % LPG) == 0) {
@@ -94,6 +118,7 @@ scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
                 reinterpret_cast<uint8_t*>(scales)[gi] = (uint8_t)q;
             }
         }
+      }
     }
     if (bad) atomicOr(&ctrl->nonfinite, 1u);
 }
