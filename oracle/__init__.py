@@ -230,6 +230,19 @@ def output_error(W, codes, s, ts, Tb, I, mode, g) -> float:
                                            C.c_int64(N), C.c_int64(K), C.c_int(mode), C.c_int(g)))
 
 
+def prescale(W, a, I=None):
+    """Per-input-channel scaling before the fit (Sec. 4, combining with AWQ): returns
+    (bf16 bits of w * a_k, I_k / a_k^2 or None)."""
+    W = _u16(W)
+    N, K = W.shape
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    Wo = np.empty_like(W)
+    Io = None if I is None else np.empty(K, dtype=np.float32)
+    Ii = None if I is None else np.ascontiguousarray(I, dtype=np.float32)
+    lib().oracle_prescale(_p(W), C.c_int64(N), C.c_int64(K), C.c_int64(K), _p(a), _p(Wo), C.c_int64(K), _p(Ii), _p(Io))
+    return Wo, Io
+
+
 def pack_sigma_bits(sigma) -> np.ndarray:
     """Alg. 1 line 20 for S < g: sigma [N x K/S] -> bits uint8 [N x K/(8 S)], group j of a row in bit
     j % 8 of byte j // 8."""

@@ -22,6 +22,8 @@
  *   oracle_pack           Alg. 1 lines 18-19, Eq. 6
  *   oracle_apply_sigma    Alg. 1 line 20   selection bit -> sign bit of the scale
  *   oracle_dequant        Eq. 5
+ *   oracle_prescale       Sec. 4 "Combining AAAC with AWQ": per-input-channel scaling of W (and the
+ *                         matching importance) before the fit
  *   oracle_pack_sigma_bits, oracle_dequant_sel, oracle_output_error_sel
  *                         the same with a selection group S smaller than the scale group g
  *                         (Sec. 3.1 "granularity"): sigma stored apart, 1/S bit per weight.
@@ -583,4 +585,20 @@ double oracle_output_error_sel(const uint16_t* W, int64_t ldw, const uint8_t* co
         E += rowE;
     }
     return E;
+}
+
+/* ------------------------------------------------------------ channel scaling before the fit */
+
+/* "AWQ first scales the weights, then AAAC learns codebooks on the scaled distribution": with a
+ * positive multiplier a_k per input channel, W'[n][k] = bf16(w a_k) (one FP32 multiply, rounded to
+ * the weights' storage type) and, because the layer's input is divided by a_k in exchange,
+ * I'_k = sum_t (X[t][k] / a_k)^2 = I_k / a_k^2, formed in double and rounded once to FP32.
+ * How the a_k are found (AWQ's search) is not part of the method.  I / I_out may be NULL. */
+void oracle_prescale(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, const float* a,
+                     uint16_t* W_out, int64_t ldo, const float* I, float* I_out) {
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k)
+            W_out[n * ldo + k] = f32_to_bf16(bf16_to_f32(W[n * ldw + k]) * a[k]);
+    if (I && I_out)
+        for (int64_t k = 0; k < K; ++k) I_out[k] = (float)((double)I[k] / ((double)a[k] * (double)a[k]));
 }
