@@ -183,6 +183,22 @@ int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* si
                      void* What, int64_t ldo, void* stream);
 
 /*
+ * Per-input-channel scaling before the fit (Section 4, "Combining AAAC with AWQ": AWQ scales
+ * the weights, AAAC then learns its tables on the scaled distribution).  The multipliers a_k
+ * themselves come from the caller (AWQ's search is not part of the method).
+ *
+ *   a       in   [K] FP32, positive and finite (else AAAC_DEV_NONFINITE is OR-ed into dev_status)
+ *   W_out   out  [N][ldo] BF16: bf16_rne(fl32(w * a_k)); may be W itself (in place)
+ *   I, I_out     both NULL, or [K] FP32 in / out: I_out[k] = I[k] / a_k^2 (double, rounded once) --
+ *                the importance of the layer's input once it is divided by a_k; may alias
+ * Feed W_out and I_out to aaac_fit_layer / aaac_pack; the dequantised weights are then those of
+ * the scaled layer.  K % 8 == 0, ldw and ldo multiples of 8, 16-byte aligned W, W_out, a.
+ */
+int aaac_prescale_columns(const void* W, int64_t N, int64_t K, int64_t ldw, const float* a,
+                          void* W_out, int64_t ldo, const float* I, float* I_out,
+                          uint32_t* dev_status /* may be NULL */, void* stream);
+
+/*
  * Whole path for one layer with HOST buffers: copies W and X to the device (into ws), runs
  * aaac_act_stats, aaac_fit_layer and aaac_pack, and copies tables, scales, tensor scale,
  * codes and errors back.  Host buffers should be page-locked for the copies to be

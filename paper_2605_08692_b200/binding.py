@@ -20,7 +20,7 @@ _lib = None
 
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
-           "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel"]
+           "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns"]
 
 
 class AaacError(RuntimeError):
@@ -53,6 +53,8 @@ def lib():
         L.aaac_pack_sel.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                     C.c_size_t, vp]
         L.aaac_dequant_sel.argtypes = [vp, vp, vp, vp, vp, i64, i64, ci, ci, ci, vp, i64, vp]
+        L.aaac_prescale_columns.argtypes = [vp, i64, i64, i64, vp, vp, i64, vp, vp, vp, vp]
+        L.aaac_prescale_columns.restype = ci
         L.aaac_quantize_layer_host.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                C.c_size_t, vp]
         L.aaac_timing_begin.argtypes = [ci]
@@ -141,6 +143,13 @@ def dequant(codes, scales, tensor_scale, T01_bf16, mode, What, group=None, sel_g
         return
     _check(lib().aaac_dequant(_ptr(codes), _ptr(scales), _ptr(tensor_scale), _ptr(T01_bf16), N, K, mode,
                               group or group_of(mode), _ptr(What), What.stride(0), _stream()))
+
+
+def prescale_columns(W, a, W_out, I=None, I_out=None, dev_status=None):
+    """W_out = bf16(W * a) per input channel (in place if W_out is W); I_out = I / a^2."""
+    N, K = W.shape
+    _check(lib().aaac_prescale_columns(_ptr(W), N, K, W.stride(0), _ptr(a), _ptr(W_out), W_out.stride(0), _ptr(I),
+                                       _ptr(I_out), _ptr(dev_status), _stream()))
 
 
 def host_workspace_bytes(mode, N, K, T) -> int:

@@ -8,7 +8,7 @@ import sys
 _DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_DIR, "csrc")
 LIB = os.environ.get("AAAC_B200_LIB") or os.path.join(_DIR, "libaaac_b200.so")
-SOURCES = ["api.cu", "act_stats.cu", "scales.cu", "init.cu", "fit.cu", "pack.cu", "dequant.cu"]
+SOURCES = ["api.cu", "act_stats.cu", "scales.cu", "init.cu", "fit.cu", "pack.cu", "dequant.cu", "prescale.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "--fmad=true", "-prec-div=true", "-prec-sqrt=true", "-ftz=false"]
 

@@ -233,6 +233,17 @@ int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* si
                           static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
 
+int aaac_prescale_columns(const void* W, int64_t N, int64_t K, int64_t ldw, const float* a,
+                          void* W_out, int64_t ldo, const float* I, float* I_out,
+                          uint32_t* dev_status, void* stream) {
+    if (!W || !a || !W_out) return AAAC_ERR_NULL;
+    if ((I == nullptr) != (I_out == nullptr)) return AAAC_ERR_NULL;
+    if (N < 1 || K < 1 || K % 8 || ldw < K || ldw % 8 || ldo < K || ldo % 8) return AAAC_ERR_SHAPE;
+    if (!aligned(W, 16) || !aligned(W_out, 16) || !aligned(a, 16)) return AAAC_ERR_ALIGN;
+    return launch_prescale(static_cast<const uint16_t*>(W), N, K, ldw, a, static_cast<uint16_t*>(W_out), ldo, I, I_out,
+                           dev_status, static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
 // ---- host-buffer path ----
 
 namespace {

@@ -126,6 +126,9 @@ cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const uint8
                            const float* tensor_scale, const uint16_t* Tb, int64_t N, int64_t K, int mode,
                            uint16_t* What, int64_t ldo, cudaStream_t st);
 
+cudaError_t launch_prescale(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, const float* a, uint16_t* Wout,
+                            int64_t ldo, const float* I, float* Iout, uint32_t* dev_status, cudaStream_t st);
+
 int sm_count();
 
 }  // namespace aaac

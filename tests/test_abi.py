@@ -82,6 +82,11 @@ def test_argument_validation_happens_on_the_host(L):
     assert L.aaac_pack_sel(ok, 64, 256, 256, 0, 128, 16, ok, ok, ok, ok, ok, ok, None, None, None, ok, big, None) == 1
     assert L.aaac_dequant_sel(ok, ok, None, ok, ok, 64, 256, 0, 128, 16, ok, 256, None) == 1
     assert L.aaac_dequant_sel(ok, ok, ok, ok, ok, 64, 256, 0, 128, 64, ok, 256, None) == 2
+    # aaac_prescale_columns
+    pre = lambda **kw: L.aaac_prescale_columns(kw.get("W", ok), 64, kw.get("K", 256), 256, kw.get("a", ok), ok, 256,
+                                               kw.get("I", None), kw.get("Io", None), None, None)
+    assert pre(W=None) == 1 and pre(a=None) == 1 and pre(I=ok) == 1
+    assert pre(K=100) == 3 and pre(W=odd) == 4
     # aaac_pack / aaac_dequant
     assert L.aaac_pack(ok, 64, 256, 256, 0, 128, None, ok, ok, ok, ok, ok, None, None, ok, big, None) == 1
     assert L.aaac_pack(ok, 64, 256, 256, 1, 16, ok, ok, ok, ok, None, ok, None, None, ok, big, None) == 1

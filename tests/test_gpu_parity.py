@@ -400,6 +400,50 @@ def test_selection_group_argument_checks():
     assert torch.equal(a["codes"], b["codes"]) and torch.equal(a["scales"], b["scales"]) and a["sigma_bits"] is None
 
 
+# ------------------------------------------------------------------ channel scaling before the fit
+
+@pytest.mark.parametrize("N,K", [(1, 8), (7, 264), (130, 1024), (4096, 4096)])
+def test_prescale_columns_bit_exact(N, K):
+    W = synth.weights(N, K, 4, f"pre/{N}x{K}/W", outlier_frac=0.02)
+    X = synth.activations(32, K, 4, f"pre/{N}x{K}/X", kind="lognormal")
+    I = oracle.act_stats(X)
+    rng = np.random.default_rng(N * 1000 + K)
+    a = np.exp(rng.normal(size=K)).astype(np.float32)
+    Wo, Io = oracle.prescale(W, a, I)
+    Wd = dev_bf16(W)
+    ad = torch.from_numpy(a).to(DEV)
+    Id = torch.from_numpy(I).to(DEV)
+    out = torch.empty_like(Wd)
+    Iout = torch.empty_like(Id)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.prescale_columns(Wd, ad, out, Id, Iout, dev_status=st)
+    assert np.array_equal(host(out), Wo)
+    assert np.array_equal(host(Iout), Io)
+    assert int(st.item()) == 0
+    # in place, without the importance
+    binding.prescale_columns(Wd, ad, Wd)
+    assert np.array_equal(host(Wd), Wo)
+    # a multiplier that is not positive and finite is reported
+    ad[K // 2] = 0.0
+    binding.prescale_columns(out, ad, out, dev_status=st)
+    assert int(st.item()) & binding.DEV_NONFINITE
+
+
+def test_prescaled_layer_goes_through_the_fit_like_any_other():
+    """Scale, then fit and pack: the same as the oracle run on the oracle's scaled layer."""
+    W, X = layer(NVFP4, 96, 768, name="prefit")
+    I = oracle.act_stats(X)
+    a = np.ones(768, np.float32)
+    a[np.argsort(I)[-16:]] = 1.75
+    Wo, Io = oracle.prescale(W, a, I)
+    Wd, ad, Id = dev_bf16(W), torch.from_numpy(a).to(DEV), torch.from_numpy(I).to(DEV)
+    binding.prescale_columns(Wd, ad, Wd, Id, Id)
+    o = oracle.fit_layer(Wo, NVFP4, 16, 5, I=Io)
+    r = binding.quantize_layer(Wd, NVFP4, I=Id, n_outer=5, init=binding.INIT_QUANTILE, want_trace=True)
+    assert table_close(host(r["T01"]), o["T"])[0]
+    check_pack(Wo, NVFP4, o, r)
+
+
 # ------------------------------------------------------------------ full benchmark sizes
 
 @pytest.mark.parametrize("which", ["q_proj", "gate_proj", "down_proj"])
