@@ -26,7 +26,9 @@ namespace aaac {
 
 namespace {
 
-constexpr int kPackWarps = 12;
+// warps per block: the INT4 instance (longer shuffle reductions) gains from 16 warps at 128 registers,
+// the NVFP4 instance is faster with 12 warps and its full register count
+constexpr int pack_warps(int mode) { return mode == AAAC_INT4 ? 16 : 12; }
 constexpr int kPackRep = 16;          // one copy of the {J_low, thr} table per lane of a half-warp: no conflicts
 
 struct PackParams {
@@ -320,6 +322,7 @@ __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long lo
 template <int MODE, int SEL>
 cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t st) {
     constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kJSlots * kSlotBytes;
+    constexpr int kPackWarps = pack_warps(MODE);
     auto kern = pack_kernel<MODE, SEL, kPackWarps, kPackRep>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -339,7 +342,7 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     p.ctrl = ws.ctrl; p.part = ws.part; p.T01_f32 = T01_f32; p.T01_bf16 = T01_bf16; p.codes = codes;
     p.sigma_bits = sigma_bits;
     const int64_t slabs = (K + 255) / 256;
-    constexpr int kRowsPerItem = kRowsPerWarp * kPackWarps;
+    const int kRowsPerItem = kRowsPerWarp * pack_warps(mode);
     const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
     if (N > 0x7FFFFFFF || K > 0x7FFFFFFF || items > 0x7FFFFFFF) return cudaErrorInvalidValue;
     int64_t grid = sm_count();
