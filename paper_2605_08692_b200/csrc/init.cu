@@ -261,9 +261,16 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned lon
     }
 }
 
-// one block per slot: radix select (4 passes of 8 bits) of every request that lives in this slot.
-// The keys of a slot lie in one narrow bin, so most of them share their leading digits: equal
-// digits within a warp are counted once (match), which keeps the shared-memory atomics apart.
+// one block per slot: radix select of every request that lives in this slot.
+//  - The first kKeep * 1024 keys of the list are read once and stay in registers for every sweep;
+//    only what is beyond them is streamed from memory, eight loads in flight per thread.
+//  - The keys of a slot lie in one narrow bin, so they share their leading bits: one sweep finds
+//    the bits on which all keys agree, and only the 8-bit digits below them need a radix pass.
+//    Within a pass equal digits within a warp are counted once (match), which keeps the
+//    shared-memory atomics apart.
+//  - The two neighbours that one table entry interpolates between are consecutive ranks: the
+//    second is the first's key again, or the smallest larger key -- one sweep instead of a
+//    second selection.
 __global__ void __launch_bounds__(1024)
 quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     __shared__ uint32_t hist[256];
@@ -271,66 +278,111 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     __shared__ unsigned long long sh_k;
     __shared__ uint32_t req_slot[kQReq];
     __shared__ unsigned long long req_local[kQReq];
+    __shared__ uint32_t sh_or, sh_and, sh_cnt, sh_min;
     const uint32_t slot = blockIdx.x;
     if (slot >= ctrl->nslots) return;
     if (threadIdx.x < kQReq) {
         req_slot[threadIdx.x] = ctrl->req_slot[threadIdx.x];
         req_local[threadIdx.x] = ctrl->req_local[threadIdx.x];
     }
+    if (threadIdx.x == 0) { sh_or = 0u; sh_and = 0xFFFFFFFFu; }
     const uint32_t* keys = list + ctrl->slot_off[slot];
     const unsigned long long n = ctrl->slot_off[slot + 1] - ctrl->slot_off[slot];
     const unsigned long long n_up = (n + blockDim.x - 1) / blockDim.x * blockDim.x;
     const int lane = threadIdx.x & 31;
-    // A list of up to kKeep keys per thread is read once and kept in registers for every pass of
-    // every request of the slot; longer lists are streamed from memory in each pass.
     constexpr int kKeep = 24;
-    const bool kept = n <= (unsigned long long)kKeep * blockDim.x;
+    const unsigned long long n_keep = min(n_up, (unsigned long long)kKeep * blockDim.x);   // a multiple of the block size
     uint32_t kc[kKeep];
 #pragma unroll
     for (int u = 0; u < kKeep; ++u) {
         const unsigned long long i = threadIdx.x + (unsigned long long)u * blockDim.x;
-        kc[u] = (kept && i < n) ? keys[i] : 0u;
+        kc[u] = i < n ? keys[i] : 0u;
     }
-    // one key's vote for its digit: equal digits within a warp are counted once
-    auto vote = [&](uint32_t k, bool sel, int shift) {
-        const unsigned act = __ballot_sync(0xFFFFFFFFu, sel);
-        if (sel) {
-            const uint32_t d = (k >> shift) & 0xFFu;
-            const unsigned peers = __match_any_sync(act, d);
-            if (lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+    // f(key, valid) for every key of the list; every thread of the block makes the same calls
+    auto for_each_key = [&](auto f) {
+#pragma unroll
+        for (int u = 0; u < kKeep; ++u) {
+            if ((unsigned long long)u * blockDim.x >= n_keep) break;
+            f(kc[u], threadIdx.x + (unsigned long long)u * blockDim.x < n);
+        }
+        for (unsigned long long i0 = n_keep + threadIdx.x; i0 < n_up; i0 += 8ull * blockDim.x) {
+            uint32_t kk[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
+                kk[u] = i < n ? keys[i] : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
+                if (i >= n_up) break;
+                f(kk[u], i < n);
+            }
         }
     };
     __syncthreads();
+    {
+        uint32_t o = 0u, a = 0xFFFFFFFFu;
+        for_each_key([&](uint32_t k, bool valid) { if (valid) { o |= k; a &= k; } });
+        o = __reduce_or_sync(0xFFFFFFFFu, o);
+        a = __reduce_and_sync(0xFFFFFFFFu, a);
+        if (lane == 0) { atomicOr(&sh_or, o); atomicAnd(&sh_and, a); }
+    }
+    __syncthreads();
+    int first_shift = 24;
+    uint32_t first_prefix = 0u, first_mask = 0u;
+    if (n > 0) {
+        const uint32_t diff = sh_or ^ sh_and;
+        first_shift = diff ? ((31 - __clz(diff)) >> 3) << 3 : 0;
+        first_mask = first_shift == 24 ? 0u : ~((1u << (first_shift + 8)) - 1u);
+        first_prefix = sh_and & first_mask;
+    }
+    bool have_prev = false;                                // rank and key of the request answered last
+    unsigned long long prev_k = 0;
+    uint32_t prev_key = 0u;
     for (int q = 0; q < kQReq; ++q) {
         if (req_slot[q] != slot) continue;                 // uniform across the block
-        if (threadIdx.x == 0) { sh_prefix = 0; sh_mask = 0; sh_k = req_local[q]; }
+        if (have_prev && (req_local[q] == prev_k || req_local[q] == prev_k + 1)) {
+            // the same or the next order statistic: it equals the previous key unless every key
+            // up to that one is already counted, in which case it is the smallest larger key
+            uint32_t key = prev_key;
+            if (req_local[q] == prev_k + 1) {
+                if (threadIdx.x == 0) { sh_cnt = 0u; sh_min = 0xFFFFFFFFu; }
+                __syncthreads();
+                uint32_t c = 0u, m = 0xFFFFFFFFu;
+                for_each_key([&](uint32_t k, bool valid) {
+                    if (valid) {
+                        if (k <= prev_key) ++c;
+                        else m = min(m, k);
+                    }
+                });
+                c = __reduce_add_sync(0xFFFFFFFFu, c);
+                m = __reduce_min_sync(0xFFFFFFFFu, m);
+                if (lane == 0) { atomicAdd(&sh_cnt, c); atomicMin(&sh_min, m); }
+                __syncthreads();
+                if (req_local[q] >= (unsigned long long)sh_cnt && sh_min != 0xFFFFFFFFu) key = sh_min;
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) ctrl->rank_val[q] = key_float(key);
+            prev_k = req_local[q];
+            prev_key = key;
+            continue;
+        }
+        if (threadIdx.x == 0) { sh_prefix = first_prefix; sh_mask = first_mask; sh_k = req_local[q]; }
         __syncthreads();
-        for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int shift = first_shift; shift >= 0; shift -= 8) {
             if (threadIdx.x < 256) hist[threadIdx.x] = 0;
             __syncthreads();
             const uint32_t prefix = sh_prefix, mask = sh_mask;
-            if (kept) {
-#pragma unroll
-                for (int u = 0; u < kKeep; ++u) {
-                    if ((unsigned long long)u * blockDim.x >= n_up) break;      // uniform over the block
-                    const unsigned long long i = threadIdx.x + (unsigned long long)u * blockDim.x;
-                    vote(kc[u], i < n && (kc[u] & mask) == prefix, shift);
+            for_each_key([&](uint32_t k, bool valid) {
+                const bool sel = valid && (k & mask) == prefix;
+                const unsigned act = __ballot_sync(0xFFFFFFFFu, sel);
+                if (sel) {
+                    const uint32_t d = (k >> shift) & 0xFFu;
+                    const unsigned peers = __match_any_sync(act, d);
+                    if (lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
                 }
-            } else
-            for (unsigned long long i0 = threadIdx.x; i0 < n_up; i0 += 4ull * blockDim.x) {
-                uint32_t kk[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {               // four independent loads in flight
-                    const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
-                    kk[u] = i < n ? keys[i] : 0u;
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const unsigned long long i = i0 + (unsigned long long)u * blockDim.x;
-                    if (i >= n_up) break;                  // uniform over the block
-                    vote(kk[u], i < n && (kk[u] & mask) == prefix, shift);
-                }
-            }
+            });
             __syncthreads();
             if (threadIdx.x < 32) {
                 // digit that holds rank k: lane l owns digits 8 l .. 8 l + 7
@@ -364,6 +416,9 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
             __syncthreads();
         }
         if (threadIdx.x == 0) ctrl->rank_val[q] = key_float(sh_prefix);
+        have_prev = true;
+        prev_k = req_local[q];
+        prev_key = sh_prefix;
         __syncthreads();
     }
 }
