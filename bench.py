@@ -381,14 +381,25 @@ def main():
                 T01=torch.empty(2, 16, dtype=torch.float32).pin_memory(), Tb=torch.empty(2, 16, dtype=torch.int16).pin_memory(),
                 sc=torch.empty(N, K // 16, dtype=torch.uint8).pin_memory(), ts=torch.empty(1, dtype=torch.float32).pin_memory(),
                 codes=torch.empty(N, K // 2, dtype=torch.uint8).pin_memory(), err=torch.empty(2, dtype=torch.float64).pin_memory(),
+                status=torch.zeros(1, dtype=torch.int32).pin_memory(), stream=torch.cuda.Stream(device=dev),
                 ws=torch.empty(binding.host_workspace_bytes(mode, N, K, TOKENS), dtype=torch.uint8, device=dev)))
 
         def host_step():
+            # one stream and one workspace per layer: a layer's copies overlap the other layers' kernels
+            # (largest copy first: the last layer's kernels are what nothing overlaps)
+            cur = torch.cuda.current_stream()
+            for h in sorted(host, key=lambda h: -(h["W"].numel() + h["X"].numel())):
+                h["stream"].wait_stream(cur)
+                with torch.cuda.stream(h["stream"]):
+                    binding.quantize_layer_host_async(h["W"], h["X"], mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE,
+                                                      T01_host=h["T01"], T01_bf16_host=h["Tb"], scales_host=h["sc"],
+                                                      tensor_scale_host=h["ts"], codes_host=h["codes"],
+                                                      err_out_host=h["err"], status_host=h["status"], ws=h["ws"])
             for h in host:
-                binding.quantize_layer_host(h["W"], h["X"], mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE,
-                                            T01_host=h["T01"], T01_bf16_host=h["Tb"], scales_host=h["sc"],
-                                            tensor_scale_host=h["ts"], codes_host=h["codes"], err_out_host=h["err"],
-                                            ws=h["ws"])
+                cur.wait_stream(h["stream"])
+            cur.synchronize()                                  # the step's results are on the host
+            if any(int(h["status"].item()) for h in host):
+                raise RuntimeError("device status is set")
         for _ in range(2):
             host_step()
         barrier()

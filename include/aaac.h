@@ -214,6 +214,19 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
                              void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same without the final synchronisation: everything, the copies back included, is only
+ * enqueued on the stream, so layers issued on different streams (each with its own ws)
+ * overlap their copies and kernels.  status_host receives the device status word
+ * (AAAC_DEV_* bits) once the stream has been synchronised by the caller; it and the other host
+ * buffers must stay valid until then and should be page-locked.
+ */
+int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int mode, int group,
+                                   const void* X_host, int64_t T, int n_outer, int init,
+                                   float* T01_host, uint16_t* T01_bf16_host, void* scales_host,
+                                   float* tensor_scale_host, uint8_t* codes_host, double* err_out_host,
+                                   uint32_t* status_host, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Optional timing of the fit-rounds kernel: after aaac_timing_begin(n) the next n launches of
  * it (one per aaac_fit_layer call with n_outer > 0, covering all rounds of that call) on the
  * calling thread's device are bracketed by CUDA events on their stream;

@@ -20,7 +20,8 @@ _lib = None
 
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
-           "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns"]
+           "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
+           "aaac_quantize_layer_host_async"]
 
 
 class AaacError(RuntimeError):
@@ -57,6 +58,9 @@ def lib():
         L.aaac_prescale_columns.restype = ci
         L.aaac_quantize_layer_host.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                C.c_size_t, vp]
+        L.aaac_quantize_layer_host_async.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
+                                                     vp, C.c_size_t, vp]
+        L.aaac_quantize_layer_host_async.restype = ci
         L.aaac_timing_begin.argtypes = [ci]
         L.aaac_timing_end.argtypes = [vp, ci]
         for f in ("aaac_act_stats", "aaac_fit_layer", "aaac_pack", "aaac_dequant", "aaac_quantize_layer_host",
@@ -165,6 +169,18 @@ def quantize_layer_host(W_host, X_host, mode, *, n_outer, init, T01_host, T01_bf
                                           _ptr(T01_host), _ptr(T01_bf16_host), _ptr(scales_host),
                                           _ptr(tensor_scale_host), _ptr(codes_host), _ptr(err_out_host), _ptr(ws),
                                           ws.numel(), _stream()))
+
+
+def quantize_layer_host_async(W_host, X_host, mode, *, n_outer, init, T01_host, T01_bf16_host, scales_host,
+                              tensor_scale_host, codes_host, err_out_host, status_host, ws):
+    """As quantize_layer_host, but only enqueued on the current stream: synchronise it before
+    reading the host tensors; status_host (pinned int32[1]) then holds the device status bits."""
+    N, K = W_host.shape
+    T = X_host.shape[0]
+    _check(lib().aaac_quantize_layer_host_async(_ptr(W_host), N, K, mode, group_of(mode), _ptr(X_host), T, n_outer,
+                                                init, _ptr(T01_host), _ptr(T01_bf16_host), _ptr(scales_host),
+                                                _ptr(tensor_scale_host), _ptr(codes_host), _ptr(err_out_host),
+                                                _ptr(status_host), _ptr(ws), ws.numel(), _stream()))
 
 
 def timing_begin(max_launches: int):

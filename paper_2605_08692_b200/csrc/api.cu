@@ -281,6 +281,21 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
                              float* T01_host, uint16_t* T01_bf16_host, void* scales_host,
                              float* tensor_scale_host, uint8_t* codes_host, double* err_out_host,
                              void* ws, size_t ws_bytes, void* stream) {
+    uint32_t hstatus = 0;
+    const int rc = aaac_quantize_layer_host_async(W_host, N, K, mode, group, X_host, T, n_outer, init, T01_host,
+                                                  T01_bf16_host, scales_host, tensor_scale_host, codes_host,
+                                                  err_out_host, &hstatus, ws, ws_bytes, stream);
+    if (rc) return rc;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return AAAC_ERR_CUDA;
+    return (hstatus & AAAC_DEV_NONFINITE) ? AAAC_ERR_NONFINITE : AAAC_OK;
+}
+
+int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int mode, int group,
+                                   const void* X_host, int64_t T, int n_outer, int init,
+                                   float* T01_host, uint16_t* T01_bf16_host, void* scales_host,
+                                   float* tensor_scale_host, uint8_t* codes_host, double* err_out_host,
+                                   uint32_t* status_host, void* ws, size_t ws_bytes, void* stream) {
+    if (!status_host) return AAAC_ERR_NULL;
     if (!W_host || !X_host || !T01_host || !T01_bf16_host || !scales_host || !tensor_scale_host || !codes_host)
         return AAAC_ERR_NULL;
     if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return AAAC_ERR_MODE;
@@ -311,7 +326,6 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
                    reinterpret_cast<float*>(d + h.ts), reinterpret_cast<uint8_t*>(d + h.codes),
                    reinterpret_cast<double*>(d + h.err), nullptr, lws, lws_bytes, stream);
     if (rc) return rc;
-    uint32_t hstatus = 0;
     cudaError_t e = cudaSuccess;
     auto back = [&](void* dst, size_t off, size_t bytes) {
         if (e == cudaSuccess && dst) e = cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st);
@@ -322,9 +336,8 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
     back(T01_bf16_host, h.Tb, 2 * kM * 2);
     back(tensor_scale_host, h.ts, 4);
     back(err_out_host, h.err, 16);
-    back(&hstatus, h.status, 4);
-    if (e != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return AAAC_ERR_CUDA;
-    return (hstatus & AAAC_DEV_NONFINITE) ? AAAC_ERR_NONFINITE : AAAC_OK;
+    back(status_host, h.status, 4);
+    return e == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
 
 // ---- timing of the fit-round kernel ----

@@ -272,6 +272,25 @@ def test_host_buffer_entry_point_matches_device_path():
     assert np.array_equal(err.numpy(), host(r["err"]))
     o = oracle.fit_layer(W, NVFP4, 16, 4, X=X)
     assert table_close(T01.numpy(), o["T"])[0]
+    # the call that only enqueues: two layers on two streams, then one synchronisation
+    outs = []
+    for k in range(2):
+        st_ = torch.cuda.Stream()
+        bufs = dict(T01=torch.empty(2, 16, dtype=torch.float32).pin_memory(), Tb=torch.empty(2, 16, dtype=torch.int16).pin_memory(),
+                    sc=torch.empty(N, K // 16, dtype=torch.uint8).pin_memory(), ts=torch.empty(1, dtype=torch.float32).pin_memory(),
+                    codes=torch.empty(N, K // 2, dtype=torch.uint8).pin_memory(), err=torch.empty(2, dtype=torch.float64).pin_memory(),
+                    status=torch.ones(1, dtype=torch.int32).pin_memory(),
+                    ws=torch.empty(binding.host_workspace_bytes(NVFP4, N, K, X.shape[0]), dtype=torch.uint8, device=DEV))
+        with torch.cuda.stream(st_):
+            binding.quantize_layer_host_async(Wh, Xh, NVFP4, n_outer=4, init=binding.INIT_QUANTILE, T01_host=bufs["T01"],
+                                              T01_bf16_host=bufs["Tb"], scales_host=bufs["sc"], tensor_scale_host=bufs["ts"],
+                                              codes_host=bufs["codes"], err_out_host=bufs["err"], status_host=bufs["status"],
+                                              ws=bufs["ws"])
+        outs.append(bufs)
+    torch.cuda.synchronize()
+    for bufs in outs:
+        assert int(bufs["status"].item()) == 0
+        assert np.array_equal(bufs["codes"].numpy(), codes.numpy()) and np.array_equal(bufs["T01"].numpy(), T01.numpy())
 
 
 # ------------------------------------------------------------------ inner refinement (n_inner > 1)
