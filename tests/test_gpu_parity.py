@@ -112,6 +112,36 @@ def test_scales_and_start_tables_bit_exact(mode, N, K):
         assert int(r["status"].item()) == 0
 
 
+@pytest.mark.parametrize("mode", [INT4, NVFP4])
+@pytest.mark.parametrize("kind", ["constant", "three_values", "two_spikes_large"])
+def test_quantile_start_tables_on_degenerate_value_sets(mode, kind):
+    """Order statistics when (nearly) all normalised weights coincide: every requested rank falls
+    into one or two histogram bins, whose lists are far longer than what the selection keeps in
+    registers, all keys share all (or all but a few) bits, and neighbouring ranks have equal keys."""
+    g = 128 if mode == INT4 else 16
+    rng = np.random.default_rng(7)
+    if kind == "constant":
+        N, K = 64, 1280
+        vals = np.full((N, K), 0.5, np.float32)
+    elif kind == "three_values":
+        N, K = 96, 1024
+        vals = rng.choice(np.array([-0.25, 0.125, 0.5], np.float32), size=(N, K))
+    else:
+        N, K = 257, 4096                              # ~1 M values on a handful of distinct w~
+        vals = rng.choice(np.array([-1.0, 1.0, 0.0], np.float32), size=(N, K), p=[0.495, 0.495, 0.01])
+    W = synth.f32_to_bf16_bits(vals)
+    I = np.ones(K, np.float32)
+    s, ts = oracle.scales(W, mode, g)
+    wt = oracle.normalise(W, mode, g, s, ts)
+    want = oracle.init_quantile(wt).astype(np.float32)
+    r = run_fit(W, mode, I, 0, binding.INIT_QUANTILE)
+    assert np.array_equal(host(r["T01"]), want), (host(r["T01"]), want)
+    # and a round from there stays on the oracle's path (many duplicate entries, empty cells)
+    o = oracle.fit_layer(W, mode, g, 2, I=I)
+    r2 = run_fit(W, mode, I, 2, binding.INIT_QUANTILE)
+    assert table_close(host(r2["T01"]), o["T"])[0]
+
+
 def test_user_tables_and_nonfinite_weights():
     W, X = layer(INT4, 16, 256, name="user")
     I = oracle.act_stats(X)
