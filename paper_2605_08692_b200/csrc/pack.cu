@@ -12,13 +12,16 @@
 // double with the exact entries, so sigma equals the double-precision decision.  The interval
 // search itself is exact (rounded-down midpoints), hence so are the codes.
 //
-// Also reported: the Eq. 8 objective under the BF16 tables, sum_k I_k (w - w^)^2 in weight units,
+// Also reported: the Eq. 8 objective under the BF16 tables, sum_k I_k (w - w^)^2 in weight units
+// (per group s^2 times the group's Eq. 8 error: w - w^ = s (w~ - T) up to the 2^-23 rounding of w~),
 // the number of groups with E0 == E1 exactly (among those re-evaluated), of weights exactly
 // half-way between two different entries of their table, and of groups re-evaluated in double.
 //
-// Thread mapping as in the fit rounds: a block of NW warps takes items of 4 NW rows x 256 columns
-// in contiguous ranges, a warp 4 rows, a lane 8 adjacent columns (one 128-bit load per row, one
-// 32-bit store of 8 codes); the next item's rows are loaded while the current one is processed.
+// Thread mapping and pipeline as in the fit rounds: a block of NW warps takes items of 4 NW rows x
+// 256 columns in contiguous ranges, a warp 4 rows, a lane 8 adjacent columns (one 128-bit load per
+// row, one 32-bit store of 8 codes); a row's registers are refilled from the next item as soon as
+// it is unpacked, the lookups of row u + 1 are issued ahead of the arithmetic of row u, and the two
+// errors travel as one packed FP32 pair.
 // Error sums go through one partial per block, added in block order by the last block to finish.
 #include "lookup.cuh"
 
@@ -26,9 +29,8 @@ namespace aaac {
 
 namespace {
 
-// warps per block: the INT4 instance (longer shuffle reductions) gains from 16 warps at 128 registers,
-// the NVFP4 instance is faster with 12 warps and its full register count
-constexpr int pack_warps(int mode) { return mode == AAAC_INT4 ? 16 : 12; }
+// warps per block (both instances run without register spills at 12; 16 is no faster)
+constexpr int pack_warps(int) { return 12; }
 constexpr int kPackRep = 16;          // one copy of the {J_low, thr} table per lane of a half-warp: no conflicts
 
 struct PackParams {
@@ -46,17 +48,54 @@ struct PackParams {
     int items, per_block, nrb;
 };
 
-// Number of the row's weights that lie exactly half-way between two different entries of the
-// chosen table (rare; kept out of line so that the hot loop stays small).
-__device__ __noinline__ int count_idx_ties(const FitTables* S, Row8 r, int sg) {
-    int n = 0;
+// The rare path of a row, out of line so that the hot loop holds a single call: for the lanes that
+// ask (flags != 0) the interval of every weight is found by binary search of the breakpoint list;
+// the groups flagged kNear are decided in double (Eq. 8 as a plain double-precision loop states
+// it, the lanes of a group combined by a shuffle tree); and for every asking lane the weights that
+// lie exactly half-way between two different entries of the chosen table are counted (x equals a
+// breakpoint that is an exact midpoint of that table).  Every lane of the warp calls.
+constexpr int kNear = 1, kTieCand = 2, kFastSigma = 4;
+struct Rare8 { int J[8]; double emin; int sigma; int tie; int nties; };
+
+template <int LPG>
+__device__ __noinline__ Rare8 rare_groups(const FitTables* S, Row8 r, int flags) {
+    Rare8 out;
+    const bool need = (flags & (kNear | kTieCand)) != 0, near = (flags & kNear) != 0;
+    double e0 = 0.0, e1 = 0.0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-#pragma unroll 1
-        for (int jj = 0; jj < kNBP; ++jj)
-            if (S->bp[jj] == r.x[j] && S->src[jj] == (uint8_t)sg && S->exact[jj]) { ++n; break; }
+        int J = 0;
+        if (need) {
+#pragma unroll
+            for (int step = 16; step; step >>= 1)          // number of breakpoints below x (sorted list)
+                if (J + step <= kNBP && S->bp[J + step - 1] < r.x[j]) J += step;
+            if (near) {
+                const double2 pq = S->PQ[J];
+                const double xd = (double)r.x[j], id = (double)r.I[j];
+                const double d0 = __dsub_rn(xd, pq.x), d1 = __dsub_rn(xd, pq.y);
+                e0 = __dadd_rn(e0, __dmul_rn(id, __dmul_rn(d0, d0)));
+                e1 = __dadd_rn(e1, __dmul_rn(id, __dmul_rn(d1, d1)));
+            }
+        }
+        out.J[j] = J;
     }
-    return n;
+#pragma unroll
+    for (int s = LPG / 2; s; s >>= 1) {
+        e0 = __dadd_rn(e0, __shfl_xor_sync(0xFFFFFFFFu, e0, s));
+        e1 = __dadd_rn(e1, __shfl_xor_sync(0xFFFFFFFFu, e1, s));
+    }
+    out.sigma = near ? (int)(e1 < e0) : ((flags & kFastSigma) != 0);
+    out.tie = near && e0 == e1;
+    out.emin = out.sigma ? e1 : e0;
+    int n = 0;
+    if (need) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            for (int jj = out.J[j]; jj < kNBP && S->bp[jj] == r.x[j]; ++jj)     // the breakpoints equal to x, if any
+                if (S->src[jj] == (uint8_t)out.sigma && S->exact[jj]) { ++n; break; }
+    }
+    out.nties = n;
+    return out;
 }
 
 template <int MODE, int SEL, int NW, int REP>
@@ -104,7 +143,8 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
     const int c0 = (int)(sm_base + kLut1Bytes + lane * 8), c1 = c0 + kSlotBytes;
     constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
     constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
-    const float tmax283 = S.tmax283;
+    // near-tie bound (see fit.cu): |E0 - E1| <= g1 (E0 + E1) + g2 sum I sends the group to the double path
+    const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
 
     double Eacc = 0.0, Eout = 0.0;
     uint32_t n_sig_tie = 0, n_idx_tie = 0, n_exact = 0;
@@ -114,164 +154,202 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
     const int it0 = blockIdx.x * p.per_block;
     const int it1 = min(p.items, it0 + p.per_block);
 
-    uint4 nv[R];
-    uint32_t ns[R];           // scale bits (sign clear): E4M3 byte or BF16 pattern
-    auto load_item = [&](int slab, int rb) {
+    // Row registers of the item being processed, refilled from the next item as soon as a row has
+    // been unpacked (as in the fit rounds).
+    uint4 v[R];
+    uint32_t sc[R];           // scale bits (sign clear): E4M3 byte or BF16 pattern
+    auto load_row = [&](int u, int slab, int rb) {
         const int col0 = slab * 256 + lane * 8;
-        const int row0 = rb * kRowsPerItem + warp * R;
-        const uint16_t* wp = p.W + (size_t)row0 * (size_t)p.ldw + col0;
-        const uint32_t g0 = (uint32_t)col0 / G;
-#pragma unroll
-        for (int u = 0; u < R; ++u) {
-            const int row = row0 + u;
-            nv[u] = make_uint4(0, 0, 0, 0);
-            ns[u] = 0u;
-            if (col0 < K && row < N) {
-                nv[u] = __ldcs(reinterpret_cast<const uint4*>(wp + (size_t)u * (size_t)p.ldw));
-                const size_t gi = (size_t)row * (size_t)Gr + g0;
-                if (MODE == AAAC_NVFP4) ns[u] = reinterpret_cast<const uint8_t*>(p.scales)[gi];
-                else ns[u] = reinterpret_cast<const uint16_t*>(p.scales)[gi];
-            }
+        const int row = rb * kRowsPerItem + warp * R + u;
+        v[u] = make_uint4(0, 0, 0, 0);
+        sc[u] = 0u;
+        if (col0 < K && row < N) {
+            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
+            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+            if (MODE == AAAC_NVFP4) sc[u] = reinterpret_cast<const uint8_t*>(p.scales)[gi];
+            else sc[u] = reinterpret_cast<const uint16_t*>(p.scales)[gi];
         }
     };
 
     int cur_slab = -1;
-    float Iv[8];
-    float isum = 0.f;
+    uint64_t II[8];           // {I, I} of the lane's eight columns
+    float isum = 0.f;         // g2 * sum of I over the lane's selection group (rounded up a little)
     bool col_ok = false;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
+    for (int j = 0; j < 8; ++j) II[j] = 0ull;
 
     int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
     int nslab = slab, nrb = rb;
-    if (it0 < it1) load_item(slab, rb);
-    for (int item = it0; item < it1; ++item) {
-        uint4 v[R];
-        uint32_t sc[R];
+    if (it0 < it1) {
 #pragma unroll
-        for (int u = 0; u < R; ++u) { v[u] = nv[u]; sc[u] = ns[u]; }
+        for (int u = 0; u < R; ++u) load_row(u, slab, rb);
+    }
+    for (int item = it0; item < it1; ++item) {
         slab = nslab;
         rb = nrb;
         if (++nrb == p.nrb) { nrb = 0; ++nslab; }
-        if (item + 1 < it1) load_item(nslab, nrb);
-
+        const bool more = item + 1 < it1;
         const int col0 = slab * 256 + lane * 8;
         if (slab != cur_slab) {
             cur_slab = slab;
             col_ok = col0 < K;
             isum = 0.f;
+            float Iv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
             if (col_ok) {
                 const float4 a = __ldg(reinterpret_cast<const float4*>(p.I + col0));
                 const float4 b = __ldg(reinterpret_cast<const float4*>(p.I + col0 + 4));
                 Iv[0] = a.x; Iv[1] = a.y; Iv[2] = a.z; Iv[3] = a.w;
                 Iv[4] = b.x; Iv[5] = b.y; Iv[6] = b.z; Iv[7] = b.w;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) isum += Iv[j];
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
             }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { isum += Iv[j]; II[j] = pack2(Iv[j], Iv[j]); }
 #pragma unroll
             for (int o = LPG / 2; o; o >>= 1) isum += __shfl_xor_sync(0xFFFFFFFFu, isum, o);
-            isum *= 1.0001f;
+            isum = __fmul_ru(isum * 1.0001f, g2);
         }
         const int row0 = rb * kRowsPerItem + warp * R;
+        const int nrows = min(R, N - row0);                // rows of this warp inside the layer (may be <= 0)
 
-#pragma unroll
-        for (int u = 0; u < R; ++u) {
-            const int row = row0 + u;
-            if (row >= N) break;                            // uniform over the warp
-            const uint32_t sbits = MODE == AAAC_NVFP4 ? (sc[u] & 0x7Fu) : (sc[u] & 0x7FFFu);
-            float sval, rinv;
+        // Stages of a row, the table lookups of the next row issued ahead of the arithmetic of this one:
+        //   L1(u): w~ and the loads of {J_low, thr};   L2: slot and the loads of {P, Q};
+        //   M(u):  errors, sigma, codes, stores.
+        float eitem = 0.f, eoitem = 0.f;                   // the item's share of the two error sums (this lane's groups)
+        float x[2][8];                                     // w~
+        uint2 e1v[2][8];                                   // {J_low * 256, thr}
+        float sval[2];                                     // scale of the row's group
+        uint32_t sbits[2];
+        uint64_t pq[8];                                    // {P, Q}, packed
+        bool tcand = false;                                // some w~ equals the breakpoint of its bin
+        auto L1 = [&](int u, int b) {
+            sbits[b] = MODE == AAAC_NVFP4 ? (sc[u] & 0x7Fu) : (sc[u] & 0x7FFFu);
+            float rinv;
             if (MODE == AAAC_NVFP4) {
-                sval = slut[sbits];
-                rinv = S.rlut[sbits];
+                sval[b] = slut[sbits[b]];
+                rinv = S.rlut[sbits[b]];
             } else {
-                sval = __uint_as_float(sbits << 16);
-                rinv = col_ok ? __frcp_rn(sval) : 0.f;
+                sval[b] = __uint_as_float(sbits[b] << 16);
+                rinv = sbits[b] ? __frcp_rn(sval[b]) : 0.f;     // lanes past K hold no scale
             }
             const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-            float x[8];
-            float2 pq[8];
-            bool tcand = false;                             // some w~ equals the breakpoint of its bin
-            float e0 = 0.f, e1 = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], 64.f, kMagic)) & kBinMask;
-                const uint2 e = lds_table_u2(lut1_lane + off);
-                const float thr = __uint_as_float(e.y);
-                tcand |= (x[j] == thr);
-                pq[j] = lds_table_f2(e.x + (uint32_t)((x[j] > thr) ? c1 : c0));
-                const float u0 = __fsub_rn(x[j], pq[j].x), u1 = __fsub_rn(x[j], pq[j].y);
-                e0 = __fmaf_rn(__fmul_rn(Iv[j], u0), u0, e0);
-                e1 = __fmaf_rn(__fmul_rn(Iv[j], u1), u1, e1);
+                x[b][j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
+                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[b][j], 64.f, kMagic)) & kBinMask;
+                e1v[b][j] = lds_table_u2(lut1_lane + off);
             }
+        };
+        auto L1n = [&](int u, int b) {
+            L1(u, b);
+            if (more) load_row(u, nslab, nrb);
+        };
+        auto L2 = [&](int b) {
+            tcand = false;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float thr = __uint_as_float(e1v[b][j].y);
+                tcand |= (x[b][j] == thr);
+                pq[j] = lds_table_b64(e1v[b][j].x + (uint32_t)((x[b][j] > thr) ? c1 : c0));
+            }
+        };
+        auto M = [&](int row, int b) {
+            uint64_t e01 = 0ull;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint64_t u01 = sub2(pack2(x[b][j], x[b][j]), pq[j]);
+                e01 = fma2(mul2(II[j], u01), u01, e01);
+            }
+            float e0 = lo2(e01), e1 = hi2(e01);
 #pragma unroll
             for (int s = LPG / 2; s; s >>= 1) {
                 e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, s);
                 e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, s);
             }
             const float es = e0 + e1;
-            const float tau = 0x1p-24f * __fmaf_rn(tmax283, __fsqrt_ru(__fmul_ru(isum, es)), 16.f * es);
+            const float tau = __fmaf_ru(es, g1, isum);
             const bool near = !(fabsf(e1 - e0) > tau) && (col_ok || !(es == es));
             bool sg = e1 < e0;
-            double emin = (double)(sg ? e1 : e0);
-            if (__any_sync(0xFFFFFFFFu, near)) {
+            float emin = sg ? e1 : e0;
+            if (__any_sync(0xFFFFFFFFu, near || tcand)) {
+                // near-ties, poisoned slots and weights that sit on a breakpoint (rare, out of line)
                 Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = Iv[j]; }
-                const Exact8 ex = exact_groups<LPG>(&S, r, (int)near);
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[b][j]; r.I[j] = lo2(II[j]); }
+                const Rare8 ex = rare_groups<LPG>(&S, r, (near ? kNear : 0) | (tcand ? kTieCand : 0) | (sg ? kFastSigma : 0));
                 if (near) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) pq[j] = lds_table_f2((uint32_t)(c0 + ex.J[j] * kSlotBytes));
+                    for (int j = 0; j < 8; ++j) pq[j] = lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes));
                     sg = ex.sigma != 0;
-                    emin = ex.emin;
-                    tcand = true;                           // poisoned slots carry no breakpoint to compare with
+                    emin = (float)ex.emin;
                     if (col_ok && (lane % LPG) == 0) { ++n_exact; n_sig_tie += ex.tie; }
                 }
+                if (col_ok) n_idx_tie += ex.nties;
             }
             if (SEL != G) {
                 // selection bits apart (Algorithm 1 line 20, S < g): group j of the row in bit j % 8 of
                 // byte j / 8; a row's 256-column slab holds 16 groups, led by the even lanes
-                uint32_t b = __ballot_sync(0xFFFFFFFFu, sg) & 0x55555555u;
-                b = (b | (b >> 1)) & 0x33333333u;
-                b = (b | (b >> 2)) & 0x0F0F0F0Fu;
-                b = (b | (b >> 4)) & 0x00FF00FFu;
-                b = (b | (b >> 8)) & 0x0000FFFFu;
+                uint32_t bb = __ballot_sync(0xFFFFFFFFu, sg) & 0x55555555u;
+                bb = (bb | (bb >> 1)) & 0x33333333u;
+                bb = (bb | (bb >> 2)) & 0x0F0F0F0Fu;
+                bb = (bb | (bb >> 4)) & 0x00FF00FFu;
+                bb = (bb | (bb >> 8)) & 0x0000FFFFu;
                 if (col_ok && (lane & 15) == 0)
-                    p.sigma_bits[(size_t)row * (size_t)(K >> 7) + (uint32_t)col0 / 128u] = (uint8_t)(b >> (lane >> 1));
+                    p.sigma_bits[(size_t)row * (size_t)(K >> 7) + (uint32_t)col0 / 128u] = (uint8_t)(bb >> (lane >> 1));
             }
-            if (!col_ok) continue;
-            if ((lane % LPG) == 0) Eacc += emin;
-            // codes (Eq. 6) and the error in weight units
+            if (!col_ok) return;
+            if ((lane % LPG) == 0) {
+                // both error sums from the group's smaller error: sum I (w - w^)^2 = s^2 sum I (w~ - T)^2
+                eitem += emin;
+                eoitem = __fmaf_rn(emin, __fmul_rn(sval[b], sval[b]), eoitem);
+            }
+            // codes (Eq. 6): the entry index rides in the low mantissa bits of the chosen constant
             uint32_t word = 0;
-            float eo = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint32_t cb = __float_as_uint(sg ? pq[j].y : pq[j].x);
-                word |= (cb & kIdxMask) << (4 * j);
-                const float tv = __uint_as_float((cb + 0x8000u) & 0xFFFF0000u);   // the BF16 entry itself (c is within 8 ulp of it)
-                const float wf = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
-                const float dw = __fmaf_rn(-tv, sval, wf);
-                eo = __fmaf_rn(__fmul_rn(Iv[j], dw), dw, eo);
-            }
-            Eout += (double)eo;
-            if (tcand) {
-                Row8 r;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = 0.f; }
-                n_idx_tie += count_idx_ties(&S, r, (int)sg);
+                float cP, cQ;
+                unpack2(pq[j], cP, cQ);
+                word |= (__float_as_uint(sg ? cQ : cP) & kIdxMask) << (4 * j);
             }
             *reinterpret_cast<uint32_t*>(p.codes + (((size_t)row * (size_t)K + col0) >> 1)) = word;
             if (SEL == G && (lane % LPG) == 0) {
                 const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
                 if (MODE == AAAC_NVFP4)
-                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
+                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits[b] | (sg ? 0x80u : 0u));
                 else
-                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits | (sg ? 0x8000u : 0u));
+                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits[b] | (sg ? 0x8000u : 0u));
+            }
+        };
+
+        if (nrows == R) {
+            L1n(0, 0);
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                if (u + 1 < R) L1n(u + 1, (u + 1) & 1);
+                L2(u & 1);
+                M(row0 + u, u & 1);
+            }
+        } else {
+            // ragged last row block of the layer: row by row, then refill all rows
+            uint4 vr[R];
+            uint32_t sr[R];
+#pragma unroll
+            for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; }
+            for (int u = 0; u < nrows; ++u) {
+#pragma unroll
+                for (int t = 0; t < R; ++t)
+                    if (u == t) { v[0] = vr[t]; sc[0] = sr[t]; }
+                L1(0, 0);
+                L2(0);
+                M(row0 + u, 0);
+            }
+            if (more) {
+#pragma unroll
+                for (int t = 0; t < R; ++t) load_row(t, nslab, nrb);
             }
         }
+        Eacc += (double)eitem;
+        Eout += (double)eoitem;
     }
 
     // ---- block partial of the two error sums; integer statistics by atomics ----
