@@ -66,10 +66,19 @@ class ClockSampler:
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits", "-lms", "20",
                                        "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
+
+    def count(self) -> int:
+        """Samples written so far."""
+        try:
+            self.f.flush()
+            with open(self.f.name) as g:
+                return sum(1 for line in g if line.count(",") >= 8)
+        except OSError:
+            return 0
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
@@ -332,10 +341,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the clock sampler starts before the warm-up steps: the query tool needs longer to start than a
+    # short timed region lasts
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(warmup):
         step()
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     binding.timing_begin(args.steps * len(layers))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -346,7 +357,17 @@ def main():
     barrier()
     ms_total = e0.elapsed_time(e1)
     round_ms = binding.timing_end(args.steps * len(layers))      # one entry per fit launch (all rounds of a layer)
-    clocks = sampler.stop() if sampler else None
+    clocks = None
+    if sampler:
+        # a timed region of a few milliseconds can end before the first sample: keep the same load
+        # running, untimed, until a few samples exist (at most two seconds)
+        extra, t_end = 0, time.time() + 2.0
+        while sampler.count() < 5 and time.time() < t_end:
+            step()
+            torch.cuda.synchronize()
+            extra += 1
+        clocks = sampler.stop()
+        clocks["window"] = f"warm-up and timed steps, plus {extra} untimed steps of the same load"
     if int(status.item()) != 0:
         raise SystemExit("device status reports non-finite input")
     ms_total = sharding.max_over_ranks(ms_total, dev)
