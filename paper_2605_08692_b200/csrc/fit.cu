@@ -491,6 +491,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     }
     // block 0 clears the next pass's buffer: every block has finished reading it (it was the buffer
     // of two passes ago) before block 0 could leave the previous barrier
+    static_assert(NT >= 256 + kUsed * kLimbs, "threads 256.. of block 0 clear the next buffer");
     if (blockIdx.x == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs)
         p.acc[(size_t)((pass_no + 1u) % 3u) * (kUsed * kLimbs) + (tid - 256)] = 0ull;
 
