@@ -530,6 +530,34 @@ def test_stack_shaped_layers_full_size(name, N, K, mode, dist):
         assert np.array_equal(host(r["scales"]), o["scales"])
 
 
+def test_config5_gate_layer_nvfp4_sampled_rows():
+    """70B-shaped gate_proj (28672 x 8192) in NVFP4 g16, 30 rounds: the tensor scale needs the whole
+    layer (the oracle's scale pass is cheap), everything after it is checked on sampled rows with
+    the library's own BF16 tables, plus the properties that hold at any size."""
+    N, K, g, rounds = 28672, 8192, 16, 30
+    c = synth.scaled_layer(N, K, 256, 0, "cfg5/gate_proj", mode=NVFP4, outlier_frac=0.005, rounds=rounds)
+    W, X = c["W"], c["X"]
+    I = oracle.act_stats(X)
+    r = run_fit(W, NVFP4, I, rounds, binding.INIT_QUANTILE)
+    assert int(r["status"].item()) == 0
+    tr = host(r["trace"])[:rounds]
+    assert np.all(tr[1:] <= tr[:-1] * (1 + 1e-6)) and tr[-1] < tr[0]
+    assert np.all(np.diff(host(r["T01"]).astype(np.float64), axis=1) >= 0)
+    s_full, ts = oracle.scales(W, NVFP4, g)
+    assert host(r["tensor_scale"])[0] == ts[0]
+    rows = np.array([0, 5, 4097, 14335, 14336, 20000, 28671])
+    assert np.array_equal(host(r["scales_pos"])[rows], s_full[rows])
+    wt = oracle.normalise(np.ascontiguousarray(W[rows]), NVFP4, g, np.ascontiguousarray(s_full[rows]), ts)
+    Tb = host(r["T01_bf16"])
+    codes, sig, _, _ = oracle.pack(wt, I, g, Tb)
+    assert np.array_equal(host(r["codes"])[rows], codes)
+    signed = oracle.apply_sigma(np.ascontiguousarray(s_full[rows]), sig, NVFP4)
+    assert np.array_equal(host(r["scales"])[rows], signed)
+    What = torch.empty(N, K, dtype=torch.bfloat16, device=DEV)
+    binding.dequant(r["codes"], r["scales"], r["tensor_scale"], r["T01_bf16"], NVFP4, What)
+    assert np.array_equal(host(What)[rows], oracle.dequant(codes, signed, ts, Tb, NVFP4, g))
+
+
 def test_config5_largest_layer_sampled_rows_and_properties():
     """70B-shaped down_proj (8192 x 28672, INT4 g128, 30 rounds): too large for the oracle to fit
     in test time, so the library's run is checked by what holds at any size -- monotone objective,
