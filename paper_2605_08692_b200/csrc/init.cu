@@ -50,7 +50,7 @@ __device__ __forceinline__ float group_rinv(const void* scales, int64_t gi, floa
 // Step 1: histogram of every w~ (shared-memory counters per block, merged with integer atomics).
 // A warp takes four 256-column pieces per iteration so that four loads are in flight.
 template <int MODE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512, 3)
 quantile_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
                      const void* __restrict__ scales, const Ctrl* ctrl, uint32_t* __restrict__ hist) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
@@ -487,10 +487,10 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     const size_t sm0 = kQBins * sizeof(uint32_t);
     if (mode == AAAC_INT4) {
         if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_INT4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
-        quantile_hist_kernel<AAAC_INT4><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
+        quantile_hist_kernel<AAAC_INT4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
     } else {
         if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_NVFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
-        quantile_hist_kernel<AAAC_NVFP4><<<blocks, 256, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
+        quantile_hist_kernel<AAAC_NVFP4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
     }
     quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qprefix, ws.qslot_of_bin);
     const int blocks1 = sm_count() * 4;
