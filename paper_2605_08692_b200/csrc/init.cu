@@ -139,28 +139,47 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
         __syncthreads();
     };
 
+    // The load of iteration k + 1 is issued before iteration k is processed, so that the block
+    // barrier at the end of an iteration does not wait for memory.
+    SlabWalk it(warp0, nwarps, slabs);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    float r = 0.f;
+    bool ok = false;
+    auto fetch = [&](uint4& vv, float& rr, bool& okk) {
+        const int64_t row = it.row, col = (int64_t)it.slab * 256 + lane * 8;
+        okk = row < N && col < K;
+        vv = make_uint4(0, 0, 0, 0);
+        rr = 0.f;
+        if (okk) {
+            vv = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
+            rr = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
+        }
+        it.next();
+    };
+    fetch(v, r, ok);
     for (int64_t k = 0; k < iters; ++k) {
-        const int64_t it = warp0 + k * nwarps;
-        if (it < items) {
-            const int64_t row = it / slabs, col = (it % slabs) * 256 + lane * 8;
-            if (col < K) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
-                const float r = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint4 vn;
+        float rn;
+        bool okn;
+        fetch(vn, rn, okn);
+        if (ok) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
-                    const uint32_t s = sm_slot[qbin(x)];
-                    if (s != 0xFFu) {
-                        const uint32_t pos = atomicAdd(&nbuf, 1u);
-                        buf_key[pos] = float_key(x);
-                        buf_slot[pos] = (uint8_t)s;
-                    }
+            for (int j = 0; j < 8; ++j) {
+                const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
+                const uint32_t s = sm_slot[qbin(x)];
+                if (s != 0xFFu) {
+                    const uint32_t pos = atomicAdd(&nbuf, 1u);
+                    buf_key[pos] = float_key(x);
+                    buf_slot[pos] = (uint8_t)s;
                 }
             }
         }
         __syncthreads();
         if (nbuf > kStageCap - kStageRoom) flush();       // uniform: nbuf is read after the barrier
+        v = vn;
+        r = rn;
+        ok = okn;
     }
     flush();
 }
