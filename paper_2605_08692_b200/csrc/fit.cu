@@ -86,6 +86,7 @@ struct FitParams {
     int trace_base;               // err_trace index of this launch's first assignment pass
     unsigned bar_base;            // passes of the layer's earlier launches (the barrier count keeps growing)
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
+    int tail_item0, tail_quarters;   // items from tail_item0 on are dealt out a quarter (one row per warp) per block
 };
 
 // hi + lo += v, error-free (Knuth's two-sum in FP32; the intrinsics keep the compiler from
@@ -168,8 +169,14 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     const int N = (int)p.N, K = (int)p.K;
     const int Gr = K / G;
     const int slabs = (K + 255) >> 8;
+    // A block takes a contiguous range of whole items; what does not divide evenly (the items from
+    // tail_item0 on) is dealt out one quarter item -- one row per warp -- per block, so that the
+    // busiest block has at most a quarter item more than the others.
     const int it0 = blockIdx.x * p.per_block;
-    const int it1 = min(p.items, it0 + p.per_block);
+    const int it1 = min(p.tail_item0, it0 + p.per_block);
+    const bool has_tail = (int)blockIdx.x < p.tail_quarters;
+    const int tail_item = p.tail_item0 + ((int)blockIdx.x >> 2), tail_u = (int)blockIdx.x & 3;
+    static_assert(R == 4, "a tail quarter is one of the four rows of a warp");
 
     if (tid < 2 * kM) S.Td[tid] = p.ctrl->T[tid];
     if (MODE == AAAC_NVFP4 && tid >= 64 && tid < 192) {
@@ -247,17 +254,25 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     for (int j = 0; j < 8; ++j) II[j] = 0ull;
 
     // (slab, row block) of the current item and of the one being loaded
-    int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
+    const int n_main = max(it1 - it0, 0), n_items = n_main + (has_tail ? 1 : 0);
+    const int first = n_main > 0 ? it0 : tail_item;
+    int slab = first / p.nrb, rb = first - slab * p.nrb;
     int nslab = slab, nrb = rb;
-    if (it0 < it1) {
+    if (n_items > 0) {
 #pragma unroll
         for (int u = 0; u < R; ++u) load_row(u, slab, rb);
     }
-    for (int item = it0; item < it1; ++item) {
+    for (int i = 0; i < n_items; ++i) {
         slab = nslab;
         rb = nrb;
-        if (++nrb == p.nrb) { nrb = 0; ++nslab; }
-        const bool more = item + 1 < it1;
+        if (i + 1 < n_main) {
+            if (++nrb == p.nrb) { nrb = 0; ++nslab; }
+        } else {                                           // the tail item comes next (if any)
+            nslab = tail_item / p.nrb;
+            nrb = tail_item - nslab * p.nrb;
+        }
+        const bool more = i + 1 < n_items;
+        const bool whole = i < n_main;                     // else: row tail_u of every warp only
 
         if (slab != cur_slab) {
             cur_slab = slab;
@@ -414,7 +429,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             }
         };
 
-        if (nrows == R) {
+        if (nrows == R && whole) {
             // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
             L1n(0);
             L2();
@@ -435,7 +450,8 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             uint32_t sr[R], gr[R];
 #pragma unroll
             for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; gr[t] = INNER ? sgw[t] : 0u; }
-            for (int u = 0; u < nrows; ++u) {
+            const int ulo = whole ? 0 : tail_u, uhi = whole ? nrows : min(nrows, tail_u + 1);
+            for (int u = ulo; u < uhi; ++u) {
                 // (u is uniform over the warp; the stages read row 0 of v[] and sc[])
 #pragma unroll
                 for (int t = 0; t < R; ++t)
@@ -568,8 +584,22 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     int64_t grid = sm_count();
     if (grid > items) grid = items;
     if (grid > kMaxFitBlocks) grid = kMaxFitBlocks;
-    const int64_t per_block = (items + grid - 1) / grid;
-    grid = (items + per_block - 1) / per_block;
+    int64_t per_block = (items + grid - 1) / grid;
+    p.tail_item0 = (int)items;
+    p.tail_quarters = 0;
+    {
+        // an even number of whole items per block plus a quarter-item tail, where that is shorter for
+        // the busiest block (a tail row costs more than a quarter of a pipelined item: count it double)
+        const int64_t g = sm_count() < kMaxFitBlocks ? sm_count() : kMaxFitBlocks;
+        const int64_t whole = items / g, rest = items - whole * g;
+        if (whole >= 4 && rest > 0 && 4 * rest <= g && 2 * whole + 1 < 2 * per_block) {
+            per_block = whole;
+            p.tail_item0 = (int)(whole * g);
+            p.tail_quarters = (int)(4 * rest);
+            grid = g;
+        }
+    }
+    if (p.tail_quarters == 0) grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
     auto launch = [&](auto kind) {
