@@ -15,8 +15,10 @@ import subprocess
 import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_DIR, "aaac_oracle.c")
-_LIB = os.path.join(_DIR, "libaaac_oracle.so")
+# AAAC_ORACLE_SRC names another copy of the source (the mutation tests plant one mistake in a
+# copy and check that a pin fails); its library is built beside it.
+_SRC = os.environ.get("AAAC_ORACLE_SRC") or os.path.join(_DIR, "aaac_oracle.c")
+_LIB = (os.path.splitext(_SRC)[0] + ".so") if os.environ.get("AAAC_ORACLE_SRC") else os.path.join(_DIR, "libaaac_oracle.so")
 _lib = None
 
 INT4, NVFP4 = 0, 1

@@ -48,6 +48,10 @@
  *   - nibble order: element 2i -> low nibble of byte i     [parity unpinned]
  *   - separate selection bits (S < g): row-major, selection group j of a row in bit j mod 8 of
  *     byte j / 8 of the row's K / (8 S) bytes                [parity unpinned]
+ *   - grid start ("init to the format's grid"): T0 = the format's table, T1 = T0 moved up
+ *     half a step, the last step repeating half the last spacing   [parity unpinned by the paper:
+ *     it starts from quantiles (Eq. 9-10) only; the half-step shift is Eq. 10's offset moved
+ *     onto a grid]
  *   - argmin ties: of two equidistant entries the smaller one, of equal entries the lowest
  *     index (on an ascending table: the lowest index); sigma tie: table 0
  *   - an inner iteration (Alg. 1 lines 15-20) updates all entries of a table at once, from
@@ -415,8 +419,13 @@ double oracle_objective(const float* wt, const float* I, int64_t N, int64_t K, i
 
 /* ------------------------------------------------------------ Alg. 1 line 17 */
 
-/* double -> FP32 -> BF16, both round-to-nearest-even (the library reports FP32 tables and
- * stores their BF16 rounding); rounding is monotone, the sort is kept for form. */
+/* Alg. 1 "Round T0, T1 to BF16".  The fitted tables are reported as FP32 numbers (the value
+ * Tf) and the stored table is the BF16 rounding of that reported number, so the chain is
+ * double -> FP32 -> BF16, both round-to-nearest-even.  It differs from a direct double -> BF16
+ * rounding only when the FP32 rounding lands exactly on a BF16 half-way point, i.e. for a
+ * double within 2^-25 relative of such a point (a 2^-17 fraction of all values); the pins
+ * count how often that happens on the seeded layers.  Rounding is monotone; the sort is kept
+ * for form. */
 void oracle_round_tables(const double* T01, float* Tf, uint16_t* Tb) {
     double t[2 * M];
     for (int i = 0; i < 2 * M; ++i) {

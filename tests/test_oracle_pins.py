@@ -86,6 +86,63 @@ def test_paper_constants():
     assert abs(float(c["delta"]) - 1.0 / (2 * (M - 1))) < 1e-16
 
 
+def test_grid_start_second_table_is_the_first_moved_up_half_a_step():
+    """The grid start's T1 against values written by hand from what the words fix (golden file):
+    INT4's uniform grid moved up half a step is -7.5 .. 7.5; on the E2M1 grid every entry of T1 is
+    the midpoint of two neighbours of T0 and the last step repeats half the last spacing."""
+    c = _consts()
+    t1_int4 = np.array([float(v) for v in c["grid_t1_int4"].split()])
+    t0_nv = np.array([float(v) for v in c["grid_t0_nvfp4"].split()])
+    t1_nv = np.array([float(v) for v in c["grid_t1_nvfp4"].split()])
+    assert len(t1_int4) == len(t0_nv) == len(t1_nv) == 16
+    g_int4, g_nv = oracle.init_grid(INT4), oracle.init_grid(NVFP4)
+    assert np.array_equal(g_int4[1], t1_int4)
+    assert np.array_equal(g_nv[0], t0_nv) and np.array_equal(g_nv[1], t1_nv)
+    # closed form, independent of the stored numbers: a uniform grid shifted by half its step
+    assert np.array_equal(g_int4[1], g_int4[0] + 0.5)
+    # every T1 entry but the last lies strictly between two neighbours of T0 (or on a doubled
+    # zero), at equal distance from both
+    for T0, T1 in ((g_int4[0], g_int4[1]), (g_nv[0], g_nv[1])):
+        assert np.array_equal(T1[:-1] - T0[:-1], T0[1:] - T1[:-1])
+        assert T1[-1] - T0[-1] == (T0[-1] - T0[-2]) / 2
+        assert np.all(np.diff(T1) >= 0)
+
+
+def _bf16_direct(v):
+    """double -> BF16 in one round-to-nearest-even step (normal range), in exact arithmetic:
+    v = q * 2^(e-8) with |q| in [128, 256); rint is exact and rounds half to even."""
+    v = np.asarray(v, dtype=np.float64)
+    m, e = np.frexp(v)                                     # v = m 2^e, |m| in [0.5, 1)
+    quantum = np.ldexp(1.0, e - 8)
+    r = np.rint(v / quantum) * quantum                     # exact: a multiple of the quantum
+    return (r.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def test_double_rounding_of_tables_equals_direct_rounding_on_the_seeded_layers():
+    """Alg. 1 rounds the tables to BF16; the chain here is double -> FP32 -> BF16.  It can differ
+    from double -> BF16 only next to a BF16 half-way point: counted over fitted tables, expected 0."""
+    differ = total = 0
+    for mode in (INT4, NVFP4):
+        for seed in range(4):
+            W, X, g = _small(mode, N=32, K=256, seed=seed, name=f"pin/dr{seed}")
+            for init in ("grid", "quantile"):
+                r = oracle.fit_layer(W, mode, g, 6, X=X, init=init)
+                direct = _bf16_direct(r["T"])
+                differ += int(np.sum(direct != r["T_bf16"]))
+                total += direct.size
+    assert total == 2 * 4 * 2 * 32 and differ == 0
+    # and a constructed value that the two chains do round differently: just above a BF16 half-way
+    # point, by less than half an FP32 step, so the FP32 rounding lands on the half-way point
+    v = 1.0 + 2.0 ** -8 + 2.0 ** -30
+    T = np.sort(np.concatenate([[v], np.arange(2, 33, dtype=np.float64)])).reshape(2, 16)
+    Tf, Tb = oracle.round_tables(T)
+    assert Tf[0, 0] == np.float32(1.0 + 2.0 ** -8)
+    assert Tb[0, 0] == 0x3F80                               # ties-to-even of the FP32 value: 1.0
+    assert _bf16_direct([v])[0] == 0x3F81
+    x = np.random.default_rng(5).standard_normal(4000) * 3
+    assert np.array_equal(_bf16_direct(x.astype(np.float32)), synth.f32_to_bf16_bits(x.astype(np.float32)))
+
+
 # ------------------------------------------------------------------ Eq. 7
 
 def test_act_stats_is_column_sum_of_squares():
@@ -330,6 +387,48 @@ def test_zero_rounds_fixed_grid_is_round_to_nearest():
             assert np.allclose(np.abs(rec - x), d_want, rtol=0, atol=1e-12)
         assert np.all(sig == 0)
         assert ties[0] == sig.size                        # identical tables: every group ties
+
+
+def _bf16_table(vals):
+    return synth.f32_to_bf16_bits(np.asarray(vals, dtype=np.float32))
+
+
+def test_pack_counts_weights_half_way_between_two_entries():
+    """ties[1] on hand-built tables: only the weights at exactly 0.5 sit half-way between two
+    different entries (0 and 1) of the table their group selects."""
+    far = np.arange(100, 114, dtype=np.float64)            # 14 entries nothing comes near
+    T_a = np.concatenate([[0.0, 1.0], far])                # 0.5 is its midpoint
+    T_b = np.concatenate([[0.0, 2.0], far])                # 0.5 is nearer to 0; its midpoint is 1
+    g, K, N = 16, 64, 3
+    rng = np.random.default_rng(11)
+    wt = np.full((N, K), 0.25, dtype=np.float32)
+    half = rng.random((N, K)) < 0.3
+    wt[half] = 0.5
+    I = rng.uniform(0.5, 2.0, K).astype(np.float32)
+    # identical tables: every group ties in selection, table 0 is used, the half-way weights count
+    codes, sig, E, ties = oracle.pack(wt, I, g, _bf16_table(np.stack([T_a, T_a])))
+    assert int(ties[0]) == sig.size and np.all(sig == 0)
+    assert int(ties[1]) == int(half.sum())
+    nib = np.stack([codes & 15, codes >> 4], axis=2).reshape(wt.shape)
+    assert np.all(nib == 0)                                # 0.25 is nearest to 0; the tie at 0.5 goes to the smaller entry
+    # table 1 = T_a wins exactly in the groups that hold a weight equal to 1 (error 0 against 1
+    # under T_b); elsewhere the errors are equal and table 0 = T_b stays, under which 0.5 is no tie
+    wt2 = wt.copy()
+    ones = np.zeros((N, K // g), dtype=bool)
+    ones[0, 1] = ones[2, 0] = ones[2, 3] = True
+    for n, j in zip(*np.nonzero(ones)):
+        wt2[n, j * g + 5] = 1.0
+        half[n, j * g + 5] = False
+    codes, sig, E, ties = oracle.pack(wt2, I, g, _bf16_table(np.stack([T_b, T_a])))
+    assert np.array_equal(sig.astype(bool), ones)
+    want = sum(int(half[n, j * g:(j + 1) * g].sum()) for n, j in zip(*np.nonzero(ones)))
+    assert want > 0 and int(ties[1]) == want
+    assert int(ties[0]) == int((~ones).sum())
+    # a duplicated entry is not "two different entries": a weight on it does not count
+    T_d = np.concatenate([[0.0, 1.0, 1.0], far[:-1]])
+    wt3 = np.full((1, g), 1.0, dtype=np.float32)
+    codes, sig, E, ties = oracle.pack(wt3, I[:g], g, _bf16_table(np.stack([T_d, T_d])))
+    assert int(ties[1]) == 0 and np.all((codes & 15) == 1) and np.all((codes >> 4) == 1)
 
 
 # ------------------------------------------------------------------ sign bit, dequant
