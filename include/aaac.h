@@ -8,7 +8,10 @@
  *
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns every
- *     buffer; the library allocates nothing and keeps no per-call state.
+ *     buffer; the library allocates no device memory and keeps no per-call state, except for
+ *     three process-wide diagnostics / conveniences that are documented where they are declared:
+ *     the event table of aaac_timing_begin / aaac_timing_end, the launch counter of
+ *     aaac_launch_count, and the built-in scratch array of aaac_act_stats_noalloc.
  *   - W is [N x K] row-major BF16 (N = output rows, K = input channels, y = x W^T, Sec. 3.1),
  *     leading dimension ldw (elements).  Groups are g contiguous elements of a row.
  *     X is [T x K] row-major BF16 calibration activations, leading dimension ldx.
@@ -18,8 +21,12 @@
  *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued and never synchronised:
  *     results are valid once the stream has been synchronised by the caller.
  *   - Return value: AAAC_OK or an aaac_status for argument / launch errors (checked before any
- *     work is enqueued).  Data-dependent conditions (non-finite input) are OR-ed into the
- *     optional device word `dev_status` instead; nothing traps.
+ *     work is enqueued).  Conditions that only the device sees are OR-ed into the optional
+ *     device word `dev_status` instead (AAAC_DEV_* bits); nothing traps.  AAAC_DEV_NONFINITE:
+ *     W, X or a multiplier holds Inf / NaN.  AAAC_DEV_TIMEOUT: a bounded wait between the
+ *     blocks of the fit-rounds kernel ran out (the kernel then returns early and the tables,
+ *     and whatever is packed from them, are NOT valid).  Without a dev_status word neither can
+ *     be seen by the caller; the host-buffer calls always keep one.
  *   - Alignment: W, X, codes, What 16-byte aligned; K % 8 == 0; K % g == 0; ldw, ldx, ldo
  *     multiples of 8.
  *   - ws is scratch of at least aaac_workspace_bytes(...) bytes, 256-byte aligned.  Calls
@@ -45,7 +52,8 @@ typedef enum {
     AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
     AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
     AAAC_ERR_UNIMPLEMENTED = 8, /* reserved */
-    AAAC_ERR_TOO_LARGE = 9      /* size beyond the fixed capacity of a no-allocation entry point */
+    AAAC_ERR_TOO_LARGE = 9,     /* size beyond the fixed capacity of a no-allocation entry point */
+    AAAC_ERR_TIMEOUT = 10       /* (dev_status bit AAAC_DEV_TIMEOUT) a bounded device-side wait ran out */
 } aaac_status;
 
 typedef enum { AAAC_INT4 = 0, AAAC_NVFP4 = 1 } aaac_mode;
@@ -68,7 +76,8 @@ size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
 
 /*
  * Activation importance, Eq. 7:  I[k] = sum_t X[t,k]^2.
- * Squares are exact and accumulated in double; the sum is rounded once to FP32.
+ * The squares are exact in FP32 and are added without rounding error (an FP32 value pair per
+ * column, strips combined in a fixed order in double); the sum is rounded once to FP32.
  * accumulate = 0 overwrites I; 1 adds to the existing I (FP32 add), so that the tokens can
  * be streamed in chunks.  Sets AAAC_DEV_NONFINITE if a sum is not finite.
  */
@@ -95,7 +104,9 @@ int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, i
  *   - all calls on a GPU share the array: calls that may overlap on the GPU (different
  *     streams without ordering) race on it and give wrong sums.  The array keeps the previous
  *     call's partials; every value a call reads it has first written itself, so nothing needs
- *     clearing between calls.
+ *     clearing between calls;
+ *   - the looked-up address is kept for the life of the device's primary context; after a
+ *     cudaDeviceReset the library must be reloaded before this entry point is used again.
  */
 int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
                            uint32_t* dev_status /* may be NULL */, void* stream);
@@ -141,8 +152,11 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
  *   stats     out  [4] uint64 or NULL: {groups with E0 == E1 exactly, weights exactly half-way
  *             between two different entries of their table, groups re-evaluated in double,
  *             reserved}
- * Decisions are exact: sigma and codes equal those of a double-precision evaluation in
- * index order (near-ties of the FP32 fast path are redone in double).
+ * Decisions are those of a double-precision evaluation: the codes are exact, and a group whose
+ * FP32 errors lie within the proven rounding bound of each other is re-evaluated in double
+ * (each lane adds its eight terms in index order, the lanes of a group are then combined
+ * pairwise; against a strictly index-ordered double sum this can differ by a few 2^-53
+ * relative, far inside what "E0 == E1 exactly" can resolve on non-degenerate data).
  */
 int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
               const float* I, const float* T01_f32, uint16_t* T01_bf16,
@@ -203,8 +217,8 @@ int aaac_prescale_columns(const void* W, int64_t N, int64_t K, int64_t ldw, cons
  * aaac_act_stats, aaac_fit_layer and aaac_pack, and copies tables, scales, tensor scale,
  * codes and errors back.  Host buffers should be page-locked for the copies to be
  * asynchronous.  ws must hold aaac_host_workspace_bytes(...) bytes of DEVICE memory.
- * Synchronises the stream before returning; returns AAAC_ERR_NONFINITE if the device
- * status word was set.
+ * Synchronises the stream before returning; returns AAAC_ERR_TIMEOUT or AAAC_ERR_NONFINITE
+ * if the corresponding bit of the device status word was set (the outputs are then not valid).
  */
 size_t aaac_host_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
 int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode, int group,
@@ -235,6 +249,13 @@ int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int
  */
 int aaac_timing_begin(int max_launches);
 int aaac_timing_end(float* ms_host, int capacity);
+
+/*
+ * Number of kernels this library has launched in the calling process so far (all entry points,
+ * all devices and streams; a process-wide counter, diagnostics only).  The benchmark reports
+ * the difference across its timed region.
+ */
+unsigned long long aaac_launch_count(void);
 
 #ifdef __cplusplus
 }

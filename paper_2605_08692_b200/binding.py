@@ -14,6 +14,8 @@ import torch
 INT4, NVFP4 = 0, 1
 INIT_QUANTILE, INIT_GRID, INIT_USER = 0, 1, 2
 DEV_NONFINITE = 1
+DEV_TIMEOUT = 2          # a bounded wait between the blocks of the fit-rounds kernel ran out: results are not valid
+ERR_TIMEOUT = 10
 
 _LIB_PATH = os.environ.get("AAAC_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b200.so")
 _lib = None
@@ -21,7 +23,7 @@ _lib = None
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
-           "aaac_quantize_layer_host_async"]
+           "aaac_quantize_layer_host_async", "aaac_launch_count"]
 
 
 class AaacError(RuntimeError):
@@ -61,6 +63,8 @@ def lib():
         L.aaac_quantize_layer_host_async.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                      vp, C.c_size_t, vp]
         L.aaac_quantize_layer_host_async.restype = ci
+        L.aaac_launch_count.restype = C.c_ulonglong
+        L.aaac_launch_count.argtypes = []
         L.aaac_timing_begin.argtypes = [ci]
         L.aaac_timing_end.argtypes = [vp, ci]
         for f in ("aaac_act_stats", "aaac_fit_layer", "aaac_pack", "aaac_dequant", "aaac_quantize_layer_host",
@@ -181,6 +185,11 @@ def quantize_layer_host_async(W_host, X_host, mode, *, n_outer, init, T01_host, 
                                                 init, _ptr(T01_host), _ptr(T01_bf16_host), _ptr(scales_host),
                                                 _ptr(tensor_scale_host), _ptr(codes_host), _ptr(err_out_host),
                                                 _ptr(status_host), _ptr(ws), ws.numel(), _stream()))
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(lib().aaac_launch_count())
 
 
 def timing_begin(max_launches: int):

@@ -100,9 +100,11 @@ cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ld
     rows = (rows + kWarps - 1) / kWarps * kWarps;
     splits = (T + rows - 1) / rows;
     act_sumsq_kernel<<<dim3(bx, (unsigned)splits), kWarps * 32, 0, st>>>(X, T, K, ldx, ws.act_part, (int)rows);
+    note_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     act_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(ws.act_part, (int)splits, K, I, accumulate, dev_status);
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -170,7 +172,9 @@ extern "C" int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64
     // every partial that the second kernel reads is written by the first: nothing has to be cleared
     act_sumsq_kernel<<<dim3(bx, (unsigned)splits), kWarps * 32, 0, st>>>(static_cast<const uint16_t*>(X), T, K, ldx,
                                                                         part, (int)rows);
+    note_launch();
     if (cudaGetLastError() != cudaSuccess) return AAAC_ERR_CUDA;
     act_final_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(part, (int)splits, K, I, accumulate, dev_status);
+    note_launch();
     return cudaGetLastError() == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }

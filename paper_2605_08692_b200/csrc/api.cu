@@ -1,4 +1,5 @@
 // C ABI of the library: argument validation, workspace carving, launch sequencing.
+#include <atomic>
 #include <mutex>
 
 #include "internal.cuh"
@@ -16,6 +17,11 @@ int sm_count() {
     }
     return cached[dev];
 }
+
+namespace {
+std::atomic<unsigned long long> g_launches{0};
+}
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 namespace {
 
@@ -96,6 +102,7 @@ const char* aaac_status_string(int status) {
         case AAAC_ERR_NONFINITE: return "input holds Inf or NaN";
         case AAAC_ERR_UNIMPLEMENTED: return "not implemented";
         case AAAC_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this no-allocation entry point";
+        case AAAC_ERR_TIMEOUT: return "a bounded wait between the blocks of a kernel ran out; results are not valid";
         default: return "unknown status";
     }
 }
@@ -287,6 +294,7 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
                                                   err_out_host, &hstatus, ws, ws_bytes, stream);
     if (rc) return rc;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (hstatus & AAAC_DEV_TIMEOUT) return AAAC_ERR_TIMEOUT;
     return (hstatus & AAAC_DEV_NONFINITE) ? AAAC_ERR_NONFINITE : AAAC_OK;
 }
 
@@ -339,6 +347,8 @@ int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int
     back(status_host, h.status, 4);
     return e == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
+
+unsigned long long aaac_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 // ---- timing of the fit-round kernel ----
 

@@ -85,6 +85,7 @@ cudaError_t launch_dequant(const uint8_t* codes, const void* scales, const uint8
         dequant_kernel<AAAC_INT4, false><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, nullptr, tensor_scale, Tb, N, K, What, ldo);
     else
         dequant_kernel<AAAC_NVFP4, false><<<(unsigned)blocks, 256, 0, st>>>(codes, scales, nullptr, tensor_scale, Tb, N, K, What, ldo);
+    note_launch();
     return cudaGetLastError();
 }
 

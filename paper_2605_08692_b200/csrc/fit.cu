@@ -560,6 +560,7 @@ cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&p};
+    note_launch();
     // cooperative: every block is resident, which the grid-wide barrier relies on
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(NW * 32), args, smem, st);
 }
@@ -627,6 +628,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
 
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st) {
     export_tables_kernel<<<1, 32, 0, st>>>(ws.ctrl, T01);
+    note_launch();
     return cudaGetLastError();
 }
 

@@ -481,6 +481,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
                         const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st) {
     if (init != AAAC_INIT_QUANTILE) {
         grid_init_kernel<<<1, 32, 0, st>>>(ws.ctrl, mode, init == AAAC_INIT_USER ? T01_user : nullptr);
+        note_launch();
         return cudaGetLastError();
     }
     // positions of the 32 quantiles, as the definition states them
@@ -501,24 +502,31 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     }
     cudaError_t e;
     set_requests_kernel<<<1, 64, 0, st>>>(ws.ctrl, rq);
+    note_launch();
     if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) return e;
     const int blocks = sm_count() * 3;
     const size_t sm0 = kQBins * sizeof(uint32_t);
     if (mode == AAAC_INT4) {
         if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_INT4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
         quantile_hist_kernel<AAAC_INT4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
+        note_launch();
     } else {
         if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_NVFP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
         quantile_hist_kernel<AAAC_NVFP4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
+        note_launch();
     }
     quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qprefix, ws.qslot_of_bin);
+    note_launch();
     const int blocks1 = sm_count() * 4;
     if (mode == AAAC_INT4)
         quantile_collect_kernel<AAAC_INT4><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qslot_of_bin, ws.qlist);
     else
         quantile_collect_kernel<AAAC_NVFP4><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qslot_of_bin, ws.qlist);
+    note_launch();
     quantile_select_kernel<<<kQReq, 1024, 0, st>>>(ws.ctrl, ws.qlist);
+    note_launch();
     quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl);
+    note_launch();
     return cudaGetLastError();
 }
 

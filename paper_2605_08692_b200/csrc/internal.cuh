@@ -130,5 +130,6 @@ cudaError_t launch_prescale(const uint16_t* W, int64_t N, int64_t K, int64_t ldw
                             int64_t ldo, const float* I, float* Iout, uint32_t* dev_status, cudaStream_t st);
 
 int sm_count();
+void note_launch(int n = 1);      // counts kernel launches (aaac_launch_count)
 
 }  // namespace aaac

@@ -405,6 +405,7 @@ cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, kPackWarps * 32, smem, st>>>(p);
+    note_launch();
     return cudaGetLastError();
 }
 
@@ -435,6 +436,7 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     else e = launch_pack_variant<AAAC_NVFP4, 16>(p, (unsigned)grid, st);
     if (e != cudaSuccess) return e;
     export_pack_kernel<<<1, 32, 0, st>>>(ws.ctrl, err_out, stats);
+    note_launch();
     return cudaGetLastError();
 }
 

@@ -67,9 +67,11 @@ cudaError_t launch_prescale(const uint16_t* W, int64_t N, int64_t K, int64_t ldw
     rows = (rows + 3) / 4 * 4;
     strips = (N + rows - 1) / rows;
     prescale_kernel<<<dim3(bx, (unsigned)strips), 256, 0, st>>>(W, N, K, ldw, a, Wout, ldo, (int)rows);
+    note_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     prescale_importance_kernel<<<(unsigned)((K + 255) / 256), 256, 0, st>>>(a, K, I, Iout, dev_status);
+    note_launch();
     return cudaGetLastError();
 }
 

@@ -134,14 +134,18 @@ cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, 
     const int blocks = sm_count() * 8;
     if (mode == AAAC_NVFP4) {
         absmax_kernel<<<blocks, 256, 0, st>>>(W, N, K, ldw, ws.ctrl);
+        note_launch();
         scales_kernel<AAAC_NVFP4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, nullptr, tensor_scale, ws.ctrl);
+        note_launch();
     } else {
         scales_kernel<AAAC_INT4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, ws.rinv, tensor_scale, ws.ctrl);
+        note_launch();
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (dev_status) {
         publish_status_kernel<<<1, 1, 0, st>>>(ws.ctrl, dev_status);
+        note_launch();
         e = cudaGetLastError();
     }
     return e;

@@ -17,7 +17,7 @@ def _run(*args):
 
 
 def test_reference_arm_prints_one_json_line():
-    r = _run("--impl", "reference", "--steps", "1", "--warmup", "0")
+    r = _run("--impl", "reference", "--steps", "1", "--warmup", "0", "--ref-seconds", "4")
     assert r.returncode == 0, r.stderr[-2000:]
     lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
     assert len(lines) == 1
@@ -29,7 +29,8 @@ def test_reference_arm_prints_one_json_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
     assert d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"]["value"] == d["value"] and d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
-    assert "workload" in d["config"]
+    assert "workload" in d["config"] and d["config"]["workload"].startswith("cfg2:")
+    assert "first rows of every layer" in d["cpu_baseline"]["sample"]      # the sample is stated
 
 
 def test_own_arm_needs_a_cuda_device():

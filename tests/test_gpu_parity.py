@@ -207,16 +207,29 @@ def check_pack(W, mode, o, r):
     return st
 
 
+def check_end_to_end_bits(r, o, label, sel=False):
+    """End to end: the library's own fit must give the oracle's BF16 tables -- the entries that
+    land on the other side of a BF16 rounding boundary are counted, printed and required to be
+    none on the seeded inputs -- and from equal tables the same packed bits follow."""
+    got, want = host(r["T01_bf16"]), o["T_bf16"]
+    differ = int(np.sum(got != want))
+    print(f"{label}: BF16 table entries that differ from the oracle's: {differ} of {want.size}")
+    assert differ == 0, f"{label}: {differ} BF16 table entries straddle a rounding boundary: {got} vs {want}"
+    assert np.array_equal(host(r["codes"]), o["codes"]), f"{label}: packed codes differ end to end"
+    if sel:
+        assert np.array_equal(host(r["sigma_bits"]), o["sigma_bits"]), f"{label}: selection bits differ end to end"
+        assert np.array_equal(host(r["scales"]), o["scales_unsigned"])
+    else:
+        assert np.array_equal(host(r["scales"]), o["scales"]), f"{label}: scales / selection bits differ end to end"
+
+
 @pytest.mark.parametrize("mode,init", [(INT4, "grid"), (INT4, "quantile"), (NVFP4, "quantile"), (NVFP4, "grid")])
 @pytest.mark.parametrize("N,K", [(3, 256), (70, 640), (257, 1024)])
 def test_fit_and_pack_small(mode, init, N, K):
     W, X = layer(mode, N, K, name=f"fit{mode}{init}/{N}x{K}")
     o, r, worst = check_fit(W, X, mode, 6, init)
     check_pack(W, mode, o, r)
-    # end to end: the library's own tables give the oracle's BF16 tables, hence the same bits
-    if np.array_equal(host(r["T01_bf16"]), o["T_bf16"]):
-        assert np.array_equal(host(r["codes"]), o["codes"])
-        assert np.array_equal(host(r["scales"]), o["scales"])
+    check_end_to_end_bits(r, o, f"small {mode} {init} {N}x{K}")
 
 
 def test_config1_end_to_end():
@@ -409,9 +422,7 @@ def check_sel16(W, X, rounds, init_name, n_inner=1):
     binding.dequant(codes, sc, ts, Tb, INT4, What, sel_group=S, sigma_bits=bits)
     assert np.array_equal(host(What), oracle.dequant_sel(o["codes"], o["scales"], o["tensor_scale"], o["T_bf16"],
                                                          o["sigma_bits"], S, INT4, g))
-    if np.array_equal(host(r["T01_bf16"]), o["T_bf16"]):
-        assert np.array_equal(host(r["codes"]), o["codes"])
-        assert np.array_equal(host(r["sigma_bits"]), o["sigma_bits"])
+    check_end_to_end_bits(r, o, f"S=16 {N}x{K} {init_name}", sel=True)
     return o, r
 
 
@@ -504,10 +515,9 @@ def test_config2_full_size(which):
     o, r, worst = check_fit(W, X, NVFP4, c["rounds"], "quantile")
     st = check_pack(W, NVFP4, o, r)
     assert st[0] == 0
-    print(f"{which}: worst table deviation {worst:.2e}, double re-evaluations {st[2]}")
-    if np.array_equal(host(r["T01_bf16"]), o["T_bf16"]):
-        assert np.array_equal(host(r["codes"]), o["codes"])
-        assert np.array_equal(host(r["scales"]), o["scales"])
+    print(f"{which}: worst table deviation {worst:.2e}, selection ties {st[0]}, half-way weights {st[1]}, "
+          f"double re-evaluations {st[2]}")
+    check_end_to_end_bits(r, o, f"cfg2 {which}")
     assert np.isclose(host(r["err"])[0], o["E_final"], rtol=1e-4)
 
 
@@ -518,75 +528,39 @@ def test_config2_full_size(which):
     ("llama8b/down_proj", 4096, 14336, INT4, "normal"),
     ("qwen7b/k_proj", 512, 3584, NVFP4, "student5"),         # configuration 4 shapes, NVFP4 g16, Student-t weights
     ("qwen7b/q_proj", 3584, 3584, NVFP4, "student5"),
+    ("llama8b/gate_proj", 14336, 4096, INT4, "normal"),      # the widest / tallest linears of both stacks
+    ("qwen7b/gate_proj", 18944, 3584, NVFP4, "student5"),
+    ("qwen7b/down_proj", 3584, 18944, NVFP4, "student5"),
 ])
 def test_stack_shaped_layers_full_size(name, N, K, mode, dist):
     """Single linears of the decoder-stack configurations, whole layer against the oracle,
     quantile init, 20 rounds."""
     c = synth.scaled_layer(N, K, 512, 0, f"stack/{name}", mode=mode, dist=dist)
     o, r, worst = check_fit(c["W"], c["X"], mode, 20, "quantile")
-    check_pack(c["W"], mode, o, r)
-    if np.array_equal(host(r["T01_bf16"]), o["T_bf16"]):
-        assert np.array_equal(host(r["codes"]), o["codes"])
-        assert np.array_equal(host(r["scales"]), o["scales"])
+    st = check_pack(c["W"], mode, o, r)
+    print(f"{name}: worst table deviation {worst:.2e}, selection ties {st[0]}, half-way weights {st[1]}, "
+          f"double re-evaluations {st[2]}")
+    assert st[0] == 0
+    check_end_to_end_bits(r, o, name)
 
 
-def test_config5_gate_layer_nvfp4_sampled_rows():
-    """70B-shaped gate_proj (28672 x 8192) in NVFP4 g16, 30 rounds: the tensor scale needs the whole
-    layer (the oracle's scale pass is cheap), everything after it is checked on sampled rows with
-    the library's own BF16 tables, plus the properties that hold at any size."""
-    N, K, g, rounds = 28672, 8192, 16, 30
-    c = synth.scaled_layer(N, K, 256, 0, "cfg5/gate_proj", mode=NVFP4, outlier_frac=0.005, rounds=rounds)
+@pytest.mark.parametrize("name,N,K,mode", [
+    ("gate_proj", 28672, 8192, NVFP4),
+    ("down_proj", 8192, 28672, INT4),
+])
+def test_config5_whole_layer(name, N, K, mode):
+    """The 70B-shaped largest layers, 30 rounds, whole layer against the oracle: fitted tables
+    and objective trace, then the pack pass and the dequantised weights bit for bit, then the
+    library's own end-to-end output.  This is the size at which the lane-private FP32 sums of the
+    fit are longest."""
+    rounds = 30
+    c = synth.scaled_layer(N, K, 256, 0, f"cfg5/{name}", mode=mode, outlier_frac=0.005, rounds=rounds)
     W, X = c["W"], c["X"]
-    I = oracle.act_stats(X)
-    r = run_fit(W, NVFP4, I, rounds, binding.INIT_QUANTILE)
+    o, r, worst = check_fit(W, X, mode, rounds, "quantile")
     assert int(r["status"].item()) == 0
-    tr = host(r["trace"])[:rounds]
-    assert np.all(tr[1:] <= tr[:-1] * (1 + 1e-6)) and tr[-1] < tr[0]
-    assert np.all(np.diff(host(r["T01"]).astype(np.float64), axis=1) >= 0)
-    s_full, ts = oracle.scales(W, NVFP4, g)
-    assert host(r["tensor_scale"])[0] == ts[0]
-    rows = np.array([0, 5, 4097, 14335, 14336, 20000, 28671])
-    assert np.array_equal(host(r["scales_pos"])[rows], s_full[rows])
-    wt = oracle.normalise(np.ascontiguousarray(W[rows]), NVFP4, g, np.ascontiguousarray(s_full[rows]), ts)
-    Tb = host(r["T01_bf16"])
-    codes, sig, _, _ = oracle.pack(wt, I, g, Tb)
-    assert np.array_equal(host(r["codes"])[rows], codes)
-    signed = oracle.apply_sigma(np.ascontiguousarray(s_full[rows]), sig, NVFP4)
-    assert np.array_equal(host(r["scales"])[rows], signed)
-    What = torch.empty(N, K, dtype=torch.bfloat16, device=DEV)
-    binding.dequant(r["codes"], r["scales"], r["tensor_scale"], r["T01_bf16"], NVFP4, What)
-    assert np.array_equal(host(What)[rows], oracle.dequant(codes, signed, ts, Tb, NVFP4, g))
-
-
-def test_config5_largest_layer_sampled_rows_and_properties():
-    """70B-shaped down_proj (8192 x 28672, INT4 g128, 30 rounds): too large for the oracle to fit
-    in test time, so the library's run is checked by what holds at any size -- monotone objective,
-    ordered tables, pack objective consistent with the last rounds -- and, given the library's own
-    BF16 tables, the oracle recomputes selection bits, codes and dequantised weights of sampled rows
-    one by one (rows are independent once the tables are fixed)."""
-    N, K, g, rounds = 8192, 28672, 128, 30
-    c = synth.scaled_layer(N, K, 256, 0, "cfg5/down_proj", mode=INT4, outlier_frac=0.005, rounds=rounds)
-    W, X = c["W"], c["X"]
-    I = oracle.act_stats(X)
-    r = run_fit(W, INT4, I, rounds, binding.INIT_QUANTILE)
-    assert int(r["status"].item()) == 0
-    T = host(r["T01"]).astype(np.float64)
-    assert np.all(np.diff(T, axis=1) >= 0)
-    tr = host(r["trace"])[:rounds]
-    assert np.all(tr[1:] <= tr[:-1] * (1 + 1e-6)) and tr[-1] < tr[0]
-    e = host(r["err"])
-    assert e[0] <= tr[-1] * 1.05                      # BF16 rounding of the tables costs little
-    rows = np.array([0, 1, 777, 4095, 4096, 6001, 8191])
-    Ws = np.ascontiguousarray(W[rows])
-    s, ts = oracle.scales(Ws, INT4, g)                # INT4 scales are per group: rows are independent
-    wt = oracle.normalise(Ws, INT4, g, s, ts)
-    Tb = host(r["T01_bf16"])
-    codes, sig, _, _ = oracle.pack(wt, I, g, Tb)
-    assert np.array_equal(host(r["codes"])[rows], codes)
-    assert np.array_equal(host(r["scales"])[rows], oracle.apply_sigma(s, sig, INT4))
-    What = torch.empty(N, K, dtype=torch.bfloat16, device=DEV)
-    binding.dequant(r["codes"], r["scales"], r["tensor_scale"], r["T01_bf16"], INT4, What)
-    want = oracle.dequant(codes, oracle.apply_sigma(s, sig, INT4), ts, Tb, INT4, g)
-    assert np.array_equal(host(What)[rows], want)
-    # on the sampled rows the fitted pair beats the fixed uniform grid it replaces (Section 3)
-    assert oracle.objective(wt, I, g, T) < oracle.objective(wt, I, g, oracle.init_grid(INT4))
+    st = check_pack(W, mode, o, r)
+    print(f"cfg5 {name}: worst table deviation {worst:.2e}, selection ties {st[0]}, half-way weights {st[1]}, "
+          f"double re-evaluations {st[2]}")
+    assert st[0] == 0
+    check_end_to_end_bits(r, o, f"cfg5 {name}")
+    assert np.isclose(host(r["err"])[0], o["E_final"], rtol=1e-4)
