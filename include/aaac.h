@@ -251,6 +251,17 @@ int aaac_timing_begin(int max_launches);
 int aaac_timing_end(float* ms_host, int capacity);
 
 /*
+ * Diagnostics for the bounded wait of the fit-rounds kernel (Algorithm 1's rounds run in one
+ * persistent kernel whose blocks wait for each other's sums once per pass; a wait that runs out
+ * sets AAAC_DEV_TIMEOUT and ends the kernel).  extra_arrivals > 0 makes every later
+ * aaac_fit_layer call of the process wait for that many more blocks than exist, so the wait must
+ * run out after spin_limit polls (0 = the default of several seconds); extra_arrivals = 0 and
+ * spin_limit = 0 restore normal operation.  For tests of the error path; process-wide, not
+ * thread-safe against concurrent aaac_fit_layer calls.
+ */
+int aaac_debug_fit_wait(int extra_arrivals, unsigned spin_limit);
+
+/*
  * Number of kernels this library has launched in the calling process so far (all entry points,
  * all devices and streams; a process-wide counter, diagnostics only).  The benchmark reports
  * the difference across its timed region.

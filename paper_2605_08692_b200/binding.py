@@ -23,7 +23,7 @@ _lib = None
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
-           "aaac_quantize_layer_host_async", "aaac_launch_count"]
+           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait"]
 
 
 class AaacError(RuntimeError):
@@ -63,6 +63,8 @@ def lib():
         L.aaac_quantize_layer_host_async.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                      vp, C.c_size_t, vp]
         L.aaac_quantize_layer_host_async.restype = ci
+        L.aaac_debug_fit_wait.argtypes = [ci, C.c_uint]
+        L.aaac_debug_fit_wait.restype = ci
         L.aaac_launch_count.restype = C.c_ulonglong
         L.aaac_launch_count.argtypes = []
         L.aaac_timing_begin.argtypes = [ci]
@@ -185,6 +187,12 @@ def quantize_layer_host_async(W_host, X_host, mode, *, n_outer, init, T01_host, 
                                                 init, _ptr(T01_host), _ptr(T01_bf16_host), _ptr(scales_host),
                                                 _ptr(tensor_scale_host), _ptr(codes_host), _ptr(err_out_host),
                                                 _ptr(status_host), _ptr(ws), ws.numel(), _stream()))
+
+
+def debug_fit_wait(extra_arrivals: int = 0, spin_limit: int = 0):
+    """Test hook: make the fit rounds' bounded wait run out (extra_arrivals > 0) after spin_limit
+    polls; (0, 0) restores normal operation."""
+    _check(lib().aaac_debug_fit_wait(extra_arrivals, spin_limit))
 
 
 def launch_count() -> int:

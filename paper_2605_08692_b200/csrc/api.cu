@@ -348,6 +348,11 @@ int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int
     return e == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
 
+int aaac_debug_fit_wait(int extra_arrivals, unsigned spin_limit) {
+    set_fit_wait(extra_arrivals, spin_limit);
+    return AAAC_OK;
+}
+
 unsigned long long aaac_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 // ---- timing of the fit-round kernel ----

@@ -1,11 +1,13 @@
 // The fit rounds (Algorithm 1 lines 6-16).  With n_inner = 1 a round is the assignment step
 // (Eq. 8) and the activation-weighted centroid update (Eq. 11) in a single pass over W, and all
 // rounds of a layer run in ONE persistent kernel (one block per SM, cooperative launch): after
-// its pass every block adds its sums, as 96-bit fixed-point integers, into 65 global accumulators,
-// the blocks meet at a grid-wide barrier, and every block reads the totals, so each holds the
-// same new tables without a second barrier or a relaunch (integer addition does not depend on
-// the order in which the blocks arrive, so the result is bitwise reproducible).  The barrier wait is bounded: if it runs out, the kernel sets
-// AAAC_DEV_TIMEOUT in the device status word and returns.
+// its pass every block adds its sums, as 96-bit fixed-point integers, into 65 global accumulators;
+// every 64-bit accumulator word also counts, in its upper 16 bits, the blocks that have added to
+// it, so a block knows that a total is complete by reading the total itself -- no separate
+// barrier, no fence between the sums and an arrival counter -- and every block ends up with the
+// same new tables without a relaunch (integer addition does not depend on the order in which the
+// blocks arrive, so the result is bitwise reproducible).  The wait for the totals is bounded: if
+// it runs out, the kernel sets AAAC_DEV_TIMEOUT in the device status word and returns.
 // With n_inner > 1 the assignment pass (which is also the first inner iteration) stores the
 // selection bits, one word per row and 256-column slab, and the remaining n_inner - 1 inner
 // iterations are passes of a second instance of the kernel that reads those bits instead of
@@ -54,9 +56,11 @@
 //     sorted; block 0 stores the Eq. 8 objective of the round (sum over groups of the smaller
 //     error) and, after the last round, the tables.
 //
-// Tables in shared memory are replicated against bank conflicts: the {J_low, thr} table REP = 16
-// times (lane l uses copy l mod 16, so the 16 lanes that share a wavefront of an 8-byte load
-// never collide), the {P, Q} table and the bins once per lane.
+// Tables in shared memory are replicated against bank conflicts: the per-bin table and the
+// {P, Q} table 16 times (lane l uses copy l mod 16, so the 16 lanes that share a wavefront of an
+// 8-byte load never collide; a bin's entry holds the address of its lower interval's {P, Q} entry
+// in the same copy, and a weight above the bin's breakpoint adds the distance to the next
+// interval's entry), the bins once per lane.
 //
 // Thread mapping.  A block of NW warps works on items of 4 NW rows x 256 columns, dealt to
 // blocks as contiguous ranges (slab-major), so every sum has a fixed order and results are
@@ -78,13 +82,15 @@ struct FitParams {
     const float* rinv;            // INT4 reciprocal scales
     const float* I;
     Ctrl* ctrl;
-    unsigned long long* acc;      // [3][kUsed][3]: fixed-point sums over the blocks, one buffer per pass in rotation
+    unsigned long long* acc;      // [3][kUsed][3] words, 128 bytes apart: fixed-point sums over the blocks, one buffer per pass in rotation
     double* err_trace;            // [n_rounds] or null
     uint32_t* dev_status;         // or null
     uint32_t* sigw;               // [N][slabs]: selection bits of a row's 256-column slab, bit = lane (n_inner > 1)
     int n_rounds;                 // passes over W in this launch
     int trace_base;               // err_trace index of this launch's first assignment pass
-    unsigned bar_base;            // passes of the layer's earlier launches (the barrier count keeps growing)
+    unsigned bar_base;            // passes of the layer's earlier launches (the sum buffers rotate per pass)
+    unsigned arrivals;            // blocks whose sums a total must hold before it is read (the grid size)
+    unsigned spin_limit;          // polls of a total before the wait is given up
     int items, per_block, nrb;    // (4 NW)-row x 256-column items, items per block, row blocks per slab
     int tail_item0, tail_quarters;   // items from tail_item0 on are dealt out a quarter (one row per warp) per block
 };
@@ -100,35 +106,44 @@ __device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
     lo = __fadd_rn(lo, err);
 }
 
-constexpr int kMaxFitBlocks = 1024;                   // grid limit: block sums are added as 32-bit limbs in 64-bit words
+constexpr int kMaxFitBlocks = 1024;                   // grid limit: block sums are added as 32-bit limbs, the arrivals counted in 16 bits
 constexpr int kLimbs = 3;                             // a sum is a 96-bit two's-complement fixed-point number
-constexpr unsigned kBarrierSpinLimit = 1u << 22;      // polls of >= 64 ns each: several seconds
+constexpr unsigned kDefaultSpinLimit = 1u << 23;      // polls of >= 32 ns each: several seconds
+constexpr int kAccStride = 16;                        // accumulator words lie 128 bytes apart: one cache line each, so that the
+                                                      // blocks' atomics on different sums do not queue behind one another
+constexpr int kAccBuffer = kUsed * kLimbs * kAccStride;   // 64-bit words of one pass's buffer
+constexpr int kCountShift = 48;                       // an accumulator word: limb sum below, arrivals above
+constexpr unsigned long long kLimbMask = (1ull << kCountShift) - 1ull;
+constexpr unsigned long long kOneArrival = 1ull << kCountShift;
+constexpr long long kTopBias = 1ll << 31;             // added to the (signed) top limb so that every block adds a non-negative number
 
-// Grid-wide barrier of a cooperative launch: block arrivals are counted in ctrl->bar, which only
-// grows during a launch.  Returns false (in every thread of the block) if the wait ran out or
-// another block has given up; the caller then leaves the kernel.
-__device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        atomicAdd(&ctrl->bar, 1u);
-        bool good = true;
-        for (unsigned spins = 0;; ++spins) {
-            unsigned seen, abort;
-            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->bar) : "memory");
-            if (seen >= target) break;
-            asm volatile("ld.relaxed.gpu.u32 %0, [%1];" : "=r"(abort) : "l"(&ctrl->abort) : "memory");
-            if (abort || spins >= kBarrierSpinLimit) {
-                atomicExch(&ctrl->abort, 1u);
-                good = false;
-                break;
-            }
-            __nanosleep(64);
-        }
-        S.is_last = good;
-    }
-    __syncthreads();
-    return S.is_last != 0;
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// process-wide knobs of the wait (aaac_debug_fit_wait): extra arrivals a total must show before it is
+// taken (0 in normal use; 1 makes every wait run out) and the poll limit
+int g_extra_arrivals = 0;
+unsigned g_spin_limit = kDefaultSpinLimit;
+
+// Near-tie groups are not decided inside the row pipeline: their lanes send the row's centred
+// terms to a spare bin slot that nobody reads, the group goes on a short per-warp list, and
+// resolve_deferred (after the pass's items, or when the list fills up) decides it in double and
+// adds its weights to the bins.  That keeps the hot loop free of the slow path, whose latency every
+// pass would otherwise pay on the warp that drew the most near-ties.
+constexpr int kDeferCap = 96;                         // list entries per warp: {row, first column of the group}
+constexpr int kBinSlots = kCells + 1;                 // [sigma][entry] and the spare slot
+constexpr int kSpareSlot = kCells;
+
+__device__ __forceinline__ void sts_u2(uint32_t addr, uint32_t a, uint32_t b) {
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" :: "r"(addr), "r"(a), "r"(b) : "memory");
 }
 
 // A launch runs passes of one kind.  kRounds: assignment passes, each also the (only) inner
@@ -137,6 +152,84 @@ __device__ bool grid_barrier(FitTables& S, Ctrl* ctrl, unsigned target) {
 // iterations with the stored selection.  With n_inner > 1 a round is one kAssignKeep launch of a
 // single pass followed by one kInner launch of n_inner - 1 passes.
 enum PassKind { kRounds = 0, kAssignKeep = 1, kInner = 2 };
+
+// Decides the listed selection groups in double (Eq. 8: each lane adds its weights' terms in index
+// order, the lanes of the group are combined pairwise; a tie goes to table 0) and adds every weight
+// to the calling lane's bins under the chosen table, with the arithmetic of the row pipeline
+// (centred term I (x - c), c the chosen entry's centre constant).  Every lane of the warp calls;
+// returns the sum of the groups' smaller errors in lane 0 (0 elsewhere).
+template <int MODE, int SEL, int KIND>
+__device__ __noinline__ double resolve_deferred(const FitTables* S, const FitParams* pp, uint32_t list_addr, int count,
+                                                uint32_t bins_lane, int lane) {
+    const FitParams& p = *pp;
+    constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
+    constexpr int WPL = SEL >= 32 ? SEL / 32 : 1;        // weights per lane
+    constexpr int ACTIVE = SEL / WPL;                    // lanes that hold weights of the group (32 or 16)
+    constexpr int LPG = SEL / 8;                         // lanes of the group in the row pipeline
+    const int K = (int)p.K, Gr = K / G, slabs = (K + 255) >> 8;
+    double esum = 0.0;
+    for (int e = 0; e < count; ++e) {
+        uint32_t urow, ucol;
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(urow), "=r"(ucol) : "r"(list_addr + (uint32_t)e * 8u));
+        const int row = (int)urow, cg = (int)ucol;
+        float xs[WPL], Is[WPL];
+        int Js[WPL];
+        double e0 = 0.0, e1 = 0.0;
+        if (lane < ACTIVE) {
+#pragma unroll
+            for (int t = 0; t < WPL; ++t) {
+                const int col = cg + lane * WPL + t;
+                const uint32_t wb = p.W[(size_t)row * (size_t)p.ldw + col];
+                const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col / G;
+                const float rinv = MODE == AAAC_NVFP4 ? S->rlut[p.scales[gi] & 0x7Fu] : __ldg(p.rinv + gi);
+                const float x = __fmul_rn(__uint_as_float(wb << 16), rinv);
+                const float iv = __ldg(p.I + col);
+                int J = 0;
+#pragma unroll
+                for (int step = 16; step; step >>= 1)      // number of breakpoints below x (sorted list)
+                    if (J + step <= kNBP && S->bp[J + step - 1] < x) J += step;
+                const double2 pq = S->PQ[J];
+                const double xd = (double)x, id = (double)iv;
+                const double d0 = __dsub_rn(xd, pq.x), d1 = __dsub_rn(xd, pq.y);
+                e0 = __dadd_rn(e0, __dmul_rn(id, __dmul_rn(d0, d0)));
+                e1 = __dadd_rn(e1, __dmul_rn(id, __dmul_rn(d1, d1)));
+                xs[t] = x; Is[t] = iv; Js[t] = J;
+            }
+        }
+#pragma unroll
+        for (int o = ACTIVE / 2; o; o >>= 1) {
+            e0 = __dadd_rn(e0, __shfl_xor_sync(0xFFFFFFFFu, e0, o));
+            e1 = __dadd_rn(e1, __shfl_xor_sync(0xFFFFFFFFu, e1, o));
+        }
+        e0 = __shfl_sync(0xFFFFFFFFu, e0, 0);
+        e1 = __shfl_sync(0xFFFFFFFFu, e1, 0);
+        const bool sg = e1 < e0;
+        if (lane < ACTIVE) {
+#pragma unroll
+            for (int t = 0; t < WPL; ++t) {
+                const float2 c2 = S->pq32[Js[t]];
+                const float c = sg ? c2.y : c2.x;
+                const uint32_t a = bins_lane + ((sg ? (uint32_t)kM : 0u) + (__float_as_uint(c) & kIdxMask)) * kSlotBytes;
+                float2 b = lds_bin(a);
+                b.x += __fmul_rn(Is[t], __fsub_rn(xs[t], c));
+                b.y += Is[t];
+                sts_bin(a, b);
+            }
+        }
+        if (lane == 0) {
+            esum += sg ? e1 : e0;
+            if (KIND == kAssignKeep) {
+                // the stored selection bits of the row's slab: bit = lane of the row pipeline
+                const uint32_t first = ((uint32_t)cg & 255u) >> 3;
+                const uint32_t mask = (LPG >= 32 ? 0xFFFFFFFFu : ((1u << LPG) - 1u)) << first;
+                uint32_t* wp = p.sigw + (size_t)row * (size_t)slabs + (cg >> 8);
+                const uint32_t old = *wp;
+                *wp = sg ? (old | mask) : (old & ~mask);
+            }
+        }
+    }
+    return esum;
+}
 
 // SEL is the selection group size S (Sec. 3.1): the weights that share one codebook choice; the
 // scale group g is fixed by the format.
@@ -149,8 +242,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     constexpr int kRowsPerItem = R * NW;
     constexpr int NT = NW * 32;
     constexpr int kLut1Bytes = REP * NB * 8;
-    constexpr int kLut2Bytes = kJSlots * kSlotBytes;
-    constexpr int kBinBytes = kCells * kSlotBytes;           // per warp
+    constexpr int kBinBytes = kBinSlots * kSlotBytes;        // per warp
     static_assert(kLut1Bytes >= NW * kPartStride * 8, "the per-warp partials reuse the first table's space");
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ FitTables S;
@@ -160,9 +252,11 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     // {P, Q} table, so a lookup there needs no further arithmetic.
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
     const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;                       // + bin * REP * 8
-    const int c0 = (int)(sm_base + kLut1Bytes + lane * 8), c1 = c0 + kSlotBytes;       // + J * 256
+    const uint32_t lut2_addr = sm_base + kLut1Bytes;                                   // the {P, Q} table
     const uint32_t bins_warp = sm_base + kLut1Bytes + kLut2Bytes + warp * kBinBytes;
     const uint32_t bins_lane = bins_warp + lane * 8;                                   // + cell * 256
+    const uint32_t spare_lane = bins_lane + kSpareSlot * kSlotBytes;                   // sink of the near-tie groups' rows
+    const uint32_t list_addr = sm_base + kLut1Bytes + kLut2Bytes + NW * kBinBytes + warp * (kDeferCap * 8);
     double* wsum = reinterpret_cast<double*>(dyn);         // [NW][kPartStride], over the first table
 
     // 32-bit index arithmetic throughout (N, K < 2^31); only the final element offsets are 64-bit
@@ -214,9 +308,17 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     constexpr float kMagic = (float)(NB / 2) + 1.5f * (float)(1 << 23) / (float)(REP * 8);
     constexpr uint32_t kBinMask = (uint32_t)(NB - 1) * (REP * 8);
 
-  for (int round = 0; round < p.n_rounds; ++round) {
-    build_tables<MODE, NW, REP, NB>(S, dyn);
     for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
+  for (int round = 0; round < p.n_rounds; ++round) {
+    const unsigned pass_no = p.bar_base + (unsigned)round;
+    // block 0 clears the buffer of the next pass: it was the buffer of two passes ago, and every block
+    // finished reading it before it added to the previous pass's buffer, whose totals block 0 has seen
+    static_assert(NT >= 256 + kUsed * kLimbs, "threads 256.. of block 0 clear the next buffer");
+    if (blockIdx.x == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs) {
+        p.acc[(size_t)((pass_no + 1u) % 3u) * kAccBuffer + (size_t)(tid - 256) * kAccStride] = 0ull;
+        __threadfence();
+    }
+    build_tables<MODE, NW, REP, NB>(S, dyn);
     // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
     // most g1 * (E0 + E1) + g2 * sum I, with kappa = 1/8 (about the usual |w~ - entry|)
     const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
@@ -247,6 +349,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     };
 
     int cur_slab = -1;
+    int ndefer = 0;           // groups on the warp's list (the same in every lane)
     uint64_t II[8];           // {I, I} of the lane's eight columns
     float isum = 0.f;         // g2 * sum of I over the lane's group (rounded up a little)
     bool col_ok = false;
@@ -304,7 +407,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         //   M(u):  errors, sigma, the centred terms and bin addresses;   B(u): bins += terms.
         float eitem = 0.f;                                 // objective of this item's groups led by this lane
         float x[8];                                        // w~ of the row in L1..M
-        uint2 e1v[8];                                      // {J_low * 256, thr}
+        uint2 e1v[8];                                      // {address of the lower interval's {P, Q} entry, thr}
         uint64_t pq[8];                                    // {P, Q}, packed
         float mt[2][8];                                    // chosen centred term I (x - c) of the rows in B / M
         uint32_t ba[2][8];                                 // its bin address
@@ -327,8 +430,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         };
         auto L2 = [&]() {
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                pq[j] = lds_table_b64(e1v[j].x + (uint32_t)((x[j] > __uint_as_float(e1v[j].y)) ? c1 : c0));
+            for (int j = 0; j < 8; ++j) pq[j] = lds_table_b64(above_addr(e1v[j].x, x[j], e1v[j].y));
         };
         auto M = [&](int row, float (&mt_o)[8], uint32_t (&ba_o)[8]) {
             if constexpr (INNER) {
@@ -348,13 +450,13 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
                 if (__any_sync(0xFFFFFFFFu, bad)) {
                     Row8 r;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); }
+                    for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); r.hint[j] = kNoHint; }
                     const Exact8 ex = exact_groups<LPG>(&S, r, (int)bad);
                     if (bad) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {
                             float cP, cQ;
-                            unpack2(lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes)), cP, cQ);
+                            unpack2(lds_table_b64(pq_entry_addr(lut2_addr, ex.J[j], lane)), cP, cQ);
                             c[j] = sg ? cQ : cP;
                             mt_o[j] = __fmul_rn(lo2(II[j]), __fsub_rn(x[j], c[j]));
                         }
@@ -369,7 +471,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             uint64_t e01 = 0ull;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint64_t u01 = sub2(pack2(x[j], x[j]), pq[j]);
+                const uint64_t u01 = diff2(x[j], pq[j]);
                 m[j] = mul2(II[j], u01);
                 e01 = fma2(m[j], u01, e01);
             }
@@ -384,39 +486,32 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             // lanes past K carry I = 0 and w~ = 0; they need the exact path only if their slot is
             // poisoned (NaN), so that no NaN reaches a bin
             const bool near = !(fabsf(e1 - e0) > tau) && (col_ok || !(es == es));
-            bool sg = e1 < e0;
+            const bool sg = e1 < e0;
             float emin = sg ? e1 : e0;
+            uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0), idx_mask = kIdxMask;
             if (__any_sync(0xFFFFFFFFu, near)) {
-                // near-ties and poisoned slots: decide in double (rare, out of line), then redo
-                // this lane's centred terms from the intervals that call has found
-                Row8 r;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); }
-                const Exact8 ex = exact_groups<LPG>(&S, r, (int)near);
-                if (near) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        pq[j] = lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes));
-                        m[j] = mul2(II[j], sub2(pack2(x[j], x[j]), pq[j]));
-                    }
-                    sg = ex.sigma != 0;
-                    emin = (float)ex.emin;
-                }
+                // near-ties and poisoned slots (rare): the group goes on the warp's list, to be decided
+                // in double by resolve_deferred; its lanes send this row's terms to the spare slot
+                const bool lead = near && col_ok && (lane % LPG) == 0;
+                const unsigned lm = __ballot_sync(0xFFFFFFFFu, lead);
+                if (lead) sts_u2(list_addr + (uint32_t)(ndefer + __popc(lm & ((1u << lane) - 1u))) * 8u, (uint32_t)row,
+                                 (uint32_t)(slab * 256 + lane * 8));
+                ndefer += __popc(lm);
+                if (near) { emin = 0.f; base = spare_lane; idx_mask = 0u; }
             }
             if (col_ok && (lane % LPG) == 0) eitem += emin;
             if (keep_sigma) {
-                const unsigned bits = __ballot_sync(0xFFFFFFFFu, sg);
+                const unsigned bits = __ballot_sync(0xFFFFFFFFu, sg);        // (the bits of listed groups are set when they are decided)
                 if (lane == 0) p.sigw[(size_t)row * (size_t)slabs + slab] = bits;
             }
             // cell = entry index (low bits of the centre constant) under the chosen table
-            const uint32_t base = bins_lane + (sg ? kM * kSlotBytes : 0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 float m0, m1, cP, cQ;
                 unpack2(m[j], m0, m1);
                 unpack2(pq[j], cP, cQ);
                 mt_o[j] = sg ? m1 : m0;
-                ba_o[j] = base + (__float_as_uint(sg ? cQ : cP) & kIdxMask) * kSlotBytes;
+                ba_o[j] = base + (__float_as_uint(sg ? cQ : cP) & idx_mask) * kSlotBytes;
             }
         };
         auto B = [&](const float (&mt_i)[8], const uint32_t (&ba_i)[8], int j0, int j1) {
@@ -467,6 +562,15 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             }
         }
         Eacc += (double)eitem;
+        if (!INNER && ndefer > kDeferCap - R * (32 / LPG)) {    // the next item could overflow the list
+            __syncwarp();
+            Eacc += resolve_deferred<MODE, SEL, KIND>(&S, &p, list_addr, ndefer, bins_lane, lane);
+            ndefer = 0;
+        }
+    }
+    if (!INNER && ndefer > 0) {
+        __syncwarp();
+        Eacc += resolve_deferred<MODE, SEL, KIND>(&S, &p, list_addr, ndefer, bins_lane, lane);
     }
    };
     pass(std::integral_constant<bool, KIND == kInner>{});
@@ -475,57 +579,91 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     //      rotated, fixed order that avoids bank conflicts); then the warps are added ----
     __syncthreads();                                       // every warp is done with the lookup tables
     {
-        float hx = 0.f, lx = 0.f, hy = 0.f, ly = 0.f;
-#pragma unroll 4
+        // four interleaved error-free chains (the additions of one chain depend on each other)
+        float hx[4] = {0.f, 0.f, 0.f, 0.f}, lx[4] = {0.f, 0.f, 0.f, 0.f}, hy[4] = {0.f, 0.f, 0.f, 0.f}, ly[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
         for (int i = 0; i < 32; ++i) {
             const float2 a = lds_bin(bins_warp + lane * kSlotBytes + ((i + lane) & 31) * 8);
-            two_sum(hx, lx, a.x);
-            two_sum(hy, ly, a.y);
+            two_sum(hx[i & 3], lx[i & 3], a.x);
+            two_sum(hy[i & 3], ly[i & 3], a.y);
         }
-        wsum[warp * kPartStride + lane] = (double)hx + (double)lx;
-        wsum[warp * kPartStride + kCells + lane] = (double)hy + (double)ly;
+        wsum[warp * kPartStride + lane] = (((double)hx[0] + (double)lx[0]) + ((double)hx[1] + (double)lx[1])) +
+                                          (((double)hx[2] + (double)lx[2]) + ((double)hx[3] + (double)lx[3]));
+        wsum[warp * kPartStride + kCells + lane] = (((double)hy[0] + (double)ly[0]) + ((double)hy[1] + (double)ly[1])) +
+                                                   (((double)hy[2] + (double)ly[2]) + ((double)hy[3] + (double)ly[3]));
+        // the warp's bins start the next pass at zero (done here, ahead of the wait for the totals)
+        __syncwarp();
+#pragma unroll 8
+        for (int b = 0; b < kCells; ++b) sts_bin(bins_lane + b * kSlotBytes, make_float2(0.f, 0.f));
     }
 #pragma unroll
     for (int s = 16; s; s >>= 1) Eacc += __shfl_xor_sync(0xFFFFFFFFu, Eacc, s);
     if (lane == 0) wsum[warp * kPartStride + 2 * kCells] = Eacc;
     __syncthreads();
-    // this block's sums go into the pass's buffer as three 32-bit limbs of a 96-bit fixed-point number
-    const unsigned pass_no = p.bar_base + (unsigned)round;
-    unsigned long long* acc = p.acc + (size_t)(pass_no % 3u) * (kUsed * kLimbs);
+    // this block's sums go into the pass's buffer as three 32-bit limbs of a 96-bit fixed-point number,
+    // each with one arrival in the word's upper bits
+    unsigned long long* acc = p.acc + (size_t)(pass_no % 3u) * kAccBuffer + (size_t)tid * (kLimbs * kAccStride);   // this thread's three words
+    const unsigned long long want = (unsigned long long)p.arrivals;
+    bool ok = true;
     if (tid < kUsed) {
-        double s = 0.0;
+        double ws_[NW];                                     // the warps' sums, added pairwise (a fixed order)
 #pragma unroll
-        for (int w = 0; w < NW; ++w) s += wsum[w * kPartStride + tid];
-        const double sd = s * S.fix_scale;
-        const double t2 = floor(sd * 0x1p-64);
+        for (int w = 0; w < NW; ++w) ws_[w] = wsum[w * kPartStride + tid];
+#pragma unroll
+        for (int stride = 1; stride < NW; stride *= 2)
+#pragma unroll
+            for (int w = 0; w + stride < NW; w += 2 * stride) ws_[w] += ws_[w + stride];
+        const double sd = ws_[0] * S.fix_scale;
+        const double t2 = floor(sd * 0x1p-64);             // in [-2^30, 2^30)
         const double r = sd - t2 * 0x1p64;                 // exact, in [0, 2^64)
         const double t1 = floor(r * 0x1p-32);
         const double t0 = floor(r - t1 * 0x1p32);
-        atomicAdd(acc + tid * kLimbs + 0, (unsigned long long)t0);
-        atomicAdd(acc + tid * kLimbs + 1, (unsigned long long)t1);
-        atomicAdd(acc + tid * kLimbs + 2, (unsigned long long)(long long)t2);
+        atomicAdd(acc + 0 * kAccStride, (unsigned long long)t0 + kOneArrival);
+        atomicAdd(acc + 1 * kAccStride, (unsigned long long)t1 + kOneArrival);
+        atomicAdd(acc + 2 * kAccStride, (unsigned long long)((long long)t2 + kTopBias) + kOneArrival);
     }
-    // block 0 clears the next pass's buffer: every block has finished reading it (it was the buffer
-    // of two passes ago) before block 0 could leave the previous barrier
-    static_assert(NT >= 256 + kUsed * kLimbs, "threads 256.. of block 0 clear the next buffer");
-    if (blockIdx.x == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs)
-        p.acc[(size_t)((pass_no + 1u) % 3u) * (kUsed * kLimbs) + (tid - 256)] = 0ull;
-
-    // ---- all blocks meet; then each reads the totals ----
-    if (!grid_barrier(S, p.ctrl, (pass_no + 1u) * gridDim.x)) {
-        if (blockIdx.x == 0 && tid == 0 && p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
-        return;
+    // ---- wait until every block's sums are in, then read the totals.  One thread of the block
+    //      polls one word (all blocks add all their words at about the same time; a crowd of
+    //      pollers on the accumulators' cache lines would hold the atomics up); after it every
+    //      thread checks the arrival counts of its own words and waits on if they are short ----
+#ifndef AAAC_FIT_POLL_ALL
+#define AAAC_FIT_POLL_ALL 0
+#endif
+#if !AAAC_FIT_POLL_ALL
+    if (tid == kUsed - 1) {
+        for (unsigned spins = 0;; ++spins) {
+            if ((ld_relaxed_u64(acc) >> kCountShift) >= want) break;
+            if (spins >= p.spin_limit || ld_relaxed_u32(&p.ctrl->abort)) { ok = false; break; }
+            __nanosleep(32);
+        }
     }
+    __syncthreads();
+#endif
     if (tid < kUsed) {
-        const unsigned long long l0 = __ldcg(acc + tid * kLimbs + 0), l1 = __ldcg(acc + tid * kLimbs + 1);
-        const long long l2 = (long long)__ldcg(acc + tid * kLimbs + 2);
-        __int128 v = ((__int128)l2 << 64) + ((__int128)l1 << 32) + (__int128)l0;
+        unsigned long long w0, w1, w2;
+        for (unsigned spins = 0;; ++spins) {
+            w0 = ld_relaxed_u64(acc + 0 * kAccStride);
+            w1 = ld_relaxed_u64(acc + 1 * kAccStride);
+            w2 = ld_relaxed_u64(acc + 2 * kAccStride);
+            if ((w0 >> kCountShift) >= want && (w1 >> kCountShift) >= want && (w2 >> kCountShift) >= want) break;
+            if (spins >= p.spin_limit || ld_relaxed_u32(&p.ctrl->abort)) { ok = false; break; }
+            __nanosleep(64);
+        }
+        const long long l2 = (long long)(w2 & kLimbMask) - (long long)gridDim.x * kTopBias;
+        __int128 v = ((__int128)l2 << 64) + ((__int128)(w1 & kLimbMask) << 32) + (__int128)(w0 & kLimbMask);
         const bool neg = v < 0;
         if (neg) v = -v;
         const double mag = (double)(unsigned long long)(v >> 64) * 0x1p64 + (double)(unsigned long long)v;
         S.tot[tid] = (neg ? -mag : mag) * S.fix_unscale;
     }
-    __syncthreads();
+    if (!__syncthreads_and(ok)) {
+        // a wait ran out (here or in another block): tell the others, report, leave
+        if (tid == 0) {
+            atomicExch(&p.ctrl->abort, 1u);
+            if (p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
+        }
+        return;
+    }
     if (tid < 2 * kM) {
         // cells of duplicate entries are empty: they keep their value
         const double sx = S.tot[tid], wt = S.tot[kCells + tid];
@@ -555,7 +693,7 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
 
 template <int MODE, int SEL, int NW, int REP, int KIND>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
-    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kJSlots * kSlotBytes + (size_t)NW * kCells * kSlotBytes;
+    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kLut2Bytes + (size_t)NW * kBinSlots * kSlotBytes + (size_t)NW * kDeferCap * 8;
     auto kern = fit_rounds_kernel<MODE, SEL, NW, REP, KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -577,6 +715,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
     p.ctrl = ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(ws.part); p.err_trace = err_trace; p.dev_status = dev_status;
     p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
+    p.spin_limit = g_spin_limit;
     p.sigw = ws.qlist;            // the quantile selection's list is free once the start tables exist
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
@@ -602,6 +741,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     }
     if (p.tail_quarters == 0) grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
+    p.arrivals = (unsigned)grid + (unsigned)g_extra_arrivals;
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
     auto launch = [&](auto kind) {
         constexpr int KIND = decltype(kind)::value;
@@ -610,7 +750,8 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
         return launch_variant<AAAC_NVFP4, 16, NW, REP, KIND>(p, (unsigned)grid, st);
     };
     // the three rotating sum buffers start at zero
-    cudaError_t em = cudaMemsetAsync(p.acc, 0, sizeof(unsigned long long) * 3 * kUsed * kLimbs, st);
+    static_assert(sizeof(unsigned long long) * 3 * kAccBuffer <= sizeof(double) * 2 * kMaxBlocks * kPartStride, "the sum buffers live in the block-partial region");
+    cudaError_t em = cudaMemsetAsync(p.acc, 0, sizeof(unsigned long long) * 3 * kAccBuffer, st);
     if (em != cudaSuccess) return em;
     if (n_inner == 1) return launch(std::integral_constant<int, kRounds>{});
     for (int outer = 0; outer < n_outer; ++outer) {
@@ -624,6 +765,11 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
         p.bar_base += (unsigned)(n_inner - 1);
     }
     return cudaSuccess;
+}
+
+void set_fit_wait(int extra_arrivals, unsigned spin_limit) {
+    g_extra_arrivals = extra_arrivals > 0 ? extra_arrivals : 0;
+    g_spin_limit = spin_limit ? spin_limit : kDefaultSpinLimit;
 }
 
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st) {

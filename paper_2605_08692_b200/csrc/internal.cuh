@@ -34,8 +34,8 @@ struct Ctrl {
     uint32_t absmax_bits;           // layer max |w| as float bits (atomicMax on non-negative floats)
     uint32_t done;                  // blocks that have written their partial this round
     uint32_t nonfinite;             // set if a non-finite weight was seen
-    uint32_t bar;                   // block arrivals at the grid barrier of the fit-rounds kernel
-    uint32_t abort;                 // set when a barrier wait ran out
+    uint32_t bar;                   // (unused)
+    uint32_t abort;                 // set when a block's wait for the totals of a pass ran out
     // quantile selection
     unsigned long long rank[kQReq]; // requested 0-based ranks (host-written via kernel args)
     double frac[2 * kM];            // interpolation fraction per table entry
@@ -131,5 +131,6 @@ cudaError_t launch_prescale(const uint16_t* W, int64_t N, int64_t K, int64_t ldw
 
 int sm_count();
 void note_launch(int n = 1);      // counts kernel launches (aaac_launch_count)
+void set_fit_wait(int extra_arrivals, unsigned spin_limit);   // knobs of the fit rounds' bounded wait (aaac_debug_fit_wait)
 
 }  // namespace aaac

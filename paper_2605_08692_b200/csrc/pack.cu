@@ -66,9 +66,13 @@ __device__ __noinline__ Rare8 rare_groups(const FitTables* S, Row8 r, int flags)
     for (int j = 0; j < 8; ++j) {
         int J = 0;
         if (need) {
+            if (r.hint[j] < (uint32_t)kNJ) {
+                J = (int)r.hint[j];
+            } else {
 #pragma unroll
-            for (int step = 16; step; step >>= 1)          // number of breakpoints below x (sorted list)
-                if (J + step <= kNBP && S->bp[J + step - 1] < r.x[j]) J += step;
+                for (int step = 16; step; step >>= 1)      // number of breakpoints below x (sorted list)
+                    if (J + step <= kNBP && S->bp[J + step - 1] < r.x[j]) J += step;
+            }
             if (near) {
                 const double2 pq = S->PQ[J];
                 const double xd = (double)r.x[j], id = (double)r.I[j];
@@ -140,7 +144,7 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
 
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
     const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;
-    const int c0 = (int)(sm_base + kLut1Bytes + lane * 8), c1 = c0 + kSlotBytes;
+    const uint32_t lut2_addr = sm_base + kLut1Bytes;                // the {P, Q} table
     constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
     constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
     // near-tie bound (see fit.cu): |E0 - E1| <= g1 (E0 + E1) + g2 sum I sends the group to the double path
@@ -217,7 +221,7 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
         //   M(u):  errors, sigma, codes, stores.
         float eitem = 0.f, eoitem = 0.f;                   // the item's share of the two error sums (this lane's groups)
         float x[2][8];                                     // w~
-        uint2 e1v[2][8];                                   // {J_low * 256, thr}
+        uint2 e1v[2][8];                                   // {address of the lower interval's {P, Q} entry, thr}
         float sval[2];                                     // scale of the row's group
         uint32_t sbits[2];
         uint64_t pq[8];                                    // {P, Q}, packed
@@ -250,14 +254,14 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
             for (int j = 0; j < 8; ++j) {
                 const float thr = __uint_as_float(e1v[b][j].y);
                 tcand |= (x[b][j] == thr);
-                pq[j] = lds_table_b64(e1v[b][j].x + (uint32_t)((x[b][j] > thr) ? c1 : c0));
+                pq[j] = lds_table_b64(above_addr(e1v[b][j].x, x[b][j], e1v[b][j].y));
             }
         };
         auto M = [&](int row, int b) {
             uint64_t e01 = 0ull;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint64_t u01 = sub2(pack2(x[b][j], x[b][j]), pq[j]);
+                const uint64_t u01 = diff2(x[b][j], pq[j]);
                 e01 = fma2(mul2(II[j], u01), u01, e01);
             }
             float e0 = lo2(e01), e1 = hi2(e01);
@@ -275,11 +279,11 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
                 // near-ties, poisoned slots and weights that sit on a breakpoint (rare, out of line)
                 Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[b][j]; r.I[j] = lo2(II[j]); }
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[b][j]; r.I[j] = lo2(II[j]); r.hint[j] = interval_hint(S, pq[j]); }
                 const Rare8 ex = rare_groups<LPG>(&S, r, (near ? kNear : 0) | (tcand ? kTieCand : 0) | (sg ? kFastSigma : 0));
                 if (near) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) pq[j] = lds_table_b64((uint32_t)(c0 + ex.J[j] * kSlotBytes));
+                    for (int j = 0; j < 8; ++j) pq[j] = lds_table_b64(pq_entry_addr(lut2_addr, ex.J[j], lane));
                     sg = ex.sigma != 0;
                     emin = (float)ex.emin;
                     if (col_ok && (lane % LPG) == 0) { ++n_exact; n_sig_tie += ex.tie; }
@@ -399,7 +403,7 @@ __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long lo
 
 template <int MODE, int SEL>
 cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t st) {
-    constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kJSlots * kSlotBytes;
+    constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kLut2Bytes;
     constexpr int kPackWarps = pack_warps(MODE);
     auto kern = pack_kernel<MODE, SEL, kPackWarps, kPackRep>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -336,6 +336,45 @@ def test_host_buffer_entry_point_matches_device_path():
         assert np.array_equal(bufs["codes"].numpy(), codes.numpy()) and np.array_equal(bufs["T01"].numpy(), T01.numpy())
 
 
+def test_fit_wait_runs_out_and_is_reported():
+    """The blocks of the fit-rounds kernel wait for each other's sums once per pass, with a poll
+    limit.  Made to run out (the totals are asked to show one more block than exists; a thousand
+    polls), every block gives up within a fraction of a millisecond, the kernel returns, the device
+    status word carries AAAC_DEV_TIMEOUT, the host-buffer call returns AAAC_ERR_TIMEOUT -- and the
+    next ordinary call on the same workspace is bit for bit what it was before."""
+    W, X = layer(NVFP4, 300, 768, T=128, name="timeout")
+    N, K = W.shape
+    Wd, Xd = dev_bf16(W), dev_bf16(X)
+    ws = binding.alloc_workspace(NVFP4, N, K, X.shape[0])
+    good = binding.quantize_layer(Wd, NVFP4, X=Xd, n_outer=3, init=binding.INIT_QUANTILE, ws=ws, want_trace=True)
+    torch.cuda.synchronize()
+    assert int(good["status"].item()) == 0
+    try:
+        binding.debug_fit_wait(1, 1000)
+        bad = binding.quantize_layer(Wd, NVFP4, X=Xd, n_outer=3, init=binding.INIT_QUANTILE, ws=ws, want_trace=True)
+        torch.cuda.synchronize()
+        assert int(bad["status"].item()) & binding.DEV_TIMEOUT
+        # the host-buffer entry point turns the status bit into an error code
+        Wh = torch.from_numpy(W.view(np.int16)).pin_memory()
+        Xh = torch.from_numpy(X.view(np.int16)).pin_memory()
+        hws = torch.empty(binding.host_workspace_bytes(NVFP4, N, K, X.shape[0]), dtype=torch.uint8, device=DEV)
+        with pytest.raises(binding.AaacError, match="status 10"):
+            binding.quantize_layer_host(Wh, Xh, NVFP4, n_outer=2, init=binding.INIT_QUANTILE,
+                                        T01_host=torch.empty(2, 16, dtype=torch.float32).pin_memory(),
+                                        T01_bf16_host=torch.empty(2, 16, dtype=torch.int16).pin_memory(),
+                                        scales_host=torch.empty(N, K // 16, dtype=torch.uint8).pin_memory(),
+                                        tensor_scale_host=torch.empty(1, dtype=torch.float32).pin_memory(),
+                                        codes_host=torch.empty(N, K // 2, dtype=torch.uint8).pin_memory(),
+                                        err_out_host=torch.empty(2, dtype=torch.float64).pin_memory(), ws=hws)
+    finally:
+        binding.debug_fit_wait(0, 0)
+    again = binding.quantize_layer(Wd, NVFP4, X=Xd, n_outer=3, init=binding.INIT_QUANTILE, ws=ws, want_trace=True)
+    torch.cuda.synchronize()
+    assert int(again["status"].item()) == 0
+    for k in ("T01", "codes", "scales", "trace", "err"):
+        assert torch.equal(again[k], good[k]), k
+
+
 # ------------------------------------------------------------------ inner refinement (n_inner > 1)
 
 @pytest.mark.parametrize("mode,init", [(INT4, "grid"), (INT4, "quantile"), (NVFP4, "quantile")])
