@@ -256,14 +256,17 @@ def run_stack(args, which, emit=True):
     Iv = {k: torch.empty(x.shape[1], dtype=torch.float32, device=dev) for k, x in X.items()}
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
+    descs = [dict(W=Ws[n], I=Iv[xin], T01=out[n]["T01"], scales=out[n]["scales"], tensor_scale=out[n]["ts"], ws=out[n]["ws"])
+             for n, N, K, xin in lin]
+
     def decoder_layer():
         for k, x in X.items():
             binding.act_stats(x, Iv[k], out["down" if k == "down" else "q"]["ws"], dev_status=status)
+        # the seven linears of a decoder layer are independent: one aaac_fit_layers call
+        binding.fit_layers(descs, mode, n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE, dev_status=status,
+                           sel_group=sel)
         for n, N, K, xin in lin:
             o = out[n]
-            binding.fit_layer(Ws[n], mode, I=Iv[xin], n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE,
-                              T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status,
-                              sel_group=sel)
             binding.pack(Ws[n], mode, I=Iv[xin], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"],
                          tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"], sel_group=sel,
                          sigma_bits=o["bits"])
@@ -273,8 +276,9 @@ def run_stack(args, which, emit=True):
     torch.cuda.synchronize()
     # kernels of one decoder layer: act_stats 2 per input; per linear absmax (NVFP4) + scales, 6 of the
     # quantile start, the fit launches, export, pack + its export
-    fit_launches = 1 if n_inner == 1 else 2 * rounds
-    launches_per_layer = 2 * len(X) + len(lin) * ((2 if mode == 1 else 1) + 6 + fit_launches + 1 + 2)
+    n0 = binding.launch_count()
+    decoder_layer()
+    launches_per_layer = binding.launch_count() - n0
     sampler = ClockSampler(0)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -291,7 +295,8 @@ def run_stack(args, which, emit=True):
             "dtype": "f32", "data": "synthetic (device-generated, one decoder layer's tensors reused for every layer)",
             "config": {"workload": f"{which}: {L} decoder layers x 7 linears (hidden {H}, kv {KV}, intermediate {FF}), "
                                    f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'} S{sel or g}, {tokens} tokens per input, quantile init, "
-                                   f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds + pack",
+                                   f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds (the seven linears of a "
+                                   f"decoder layer in one aaac_fit_layers call) + pack",
                        "linears": 7 * L, "weights": wl * L, "rounds": rounds, "n_inner": n_inner},
             "gweights_per_s_per_round": wl * L * rounds * n_inner / wall / 1e9, "clocks": clocks,
             "gpu_launches": launches_per_layer * L}
@@ -385,11 +390,15 @@ def main():
             ws=binding.alloc_workspace(mode, N, K, TOKENS, dev)))
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
+    descs = [dict(W=W, I=o["I"], T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"]) for W, o in zip(Wd, outs)]
+
     def step():
-        for W, X, o in zip(Wd, Xd, outs):
+        # the layers of a step are independent: their importances first, then scales, start tables and the
+        # 20 rounds of all of them in one aaac_fit_layers call (the rounds in one launch), then pack and dequant
+        for X, o in zip(Xd, outs):
             binding.act_stats(X, o["I"], o["ws"], dev_status=status)
-            binding.fit_layer(W, mode, I=o["I"], n_outer=ROUNDS, init=binding.INIT_QUANTILE, T01=o["T01"],
-                              scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], dev_status=status)
+        binding.fit_layers(descs, mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE, dev_status=status)
+        for W, o in zip(Wd, outs):
             binding.pack(W, mode, I=o["I"], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"], tensor_scale=o["ts"],
                          codes=o["codes"], ws=o["ws"], err_out=o["err"])
             binding.dequant(o["codes"], o["scales"], o["ts"], o["Tb"], mode, o["What"])
@@ -411,7 +420,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     reps = []
     for _ in range(REPEATS):
-        binding.timing_begin(args.steps * len(layers))
+        binding.timing_begin(args.steps)
         n0 = binding.launch_count()
         barrier()
         e0.record()
@@ -421,7 +430,7 @@ def main():
         barrier()
         launches = binding.launch_count() - n0
         ms_rep = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
-        reps.append((ms_rep, binding.timing_end(args.steps * len(layers)), launches))   # one entry per fit launch (all rounds of a layer)
+        reps.append((ms_rep, binding.timing_end(args.steps), launches))   # one entry per fit launch (all rounds of the step's layers)
     reps.sort(key=lambda r: r[0])
     ms_total, round_ms, launches = reps[len(reps) // 2]
     clocks = None
@@ -441,16 +450,15 @@ def main():
     value = sharding.job_throughput(weights_per_step, ROUNDS, ms_step, world)
 
     # roofline of the dominant kernel: algorithmic bytes of every timed fit-round launch / its device time
-    per_launch_w = []
-    for _ in range(args.steps):
-        for (N, K) in shapes:
-            per_launch_w += [N * K * ROUNDS]
+    per_launch_w = [weights_per_step * ROUNDS] * args.steps
     bytes_alg = sum(per_launch_w[:len(round_ms)]) * BYTES_PER_WEIGHT
     fit_ms = float(sum(round_ms))
     achieved = bytes_alg / (fit_ms * 1e-3) / 1e9 if fit_ms > 0 else 0.0
     peak, peak_kind = peaks()
     tpw = measured_traffic_per_weight()
-    roofline = {"kernel": "fit_rounds_kernel (one launch = the 20 k-means rounds of a layer)", "bound": "hbm",
+    roofline = {"kernel": "fit_batch_kernel (one launch = the 20 k-means rounds of the step's layers, each layer on its share "
+                          "of the blocks)" if len(layers) > 1 else "fit_rounds_kernel (one launch = the 20 k-means rounds of the layer)",
+                "bound": "hbm",
                 "binding_units": "by the ncu counters the kernel is held by the shared-memory data pipe and instruction "
                                  "issue, not by HBM; the HBM fraction is reported because it is the metric",
                 "achieved": achieved, "peak": peak,
@@ -466,7 +474,7 @@ def main():
 
     # the other stages of a step, each bracketed by events inside steps of the same rotation (so a
     # layer's data has been evicted by the other layers' before it is used again); median over steps
-    stage_names = ["act_stats", "scales+init+fit+export", "pack", "dequant"]
+    stage_names = ["act_stats", "scales+init+fit+export (layer by layer)", "pack", "dequant"]
     stage_ms = {k: [] for k in stage_names}
     split_ms = []                                               # scales + quantile init alone (fit with n_outer = 0)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(layers) * 5 * 2)]

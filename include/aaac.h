@@ -197,6 +197,41 @@ int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* si
                      void* What, int64_t ldo, void* stream);
 
 /*
+ * Algorithm 1 lines 1-16 for several layers of one format at once.  The paper processes layers
+ * independently (Sec. 3.3, "Computational cost"), so a batch is only a way of running them: the
+ * result for every layer is what aaac_fit_layer_sel gives for it, up to the rounding of the FP32
+ * partial sums (a layer's rows are dealt to a share of the GPU's blocks instead of all of them;
+ * the fitted tables agree to about 1e-7 relative and are bitwise reproducible from call to call).
+ * With n_inner = 1 the rounds of up to eight layers run in one launch, each layer on its own
+ * share of the blocks, so that the cost of a round that does not depend on the layer's size is
+ * paid once per batch and small layers do not leave most of the GPU idle; more layers, and
+ * n_inner > 1, are run in turn.  Scales, importances (from X where I is NULL) and start tables
+ * are computed per layer exactly as by aaac_fit_layer_sel.
+ *
+ *   layers   HOST array of n_layers descriptors (read before the call returns); every pointer
+ *            inside is a DEVICE pointer with the meaning, layout and alignment of the
+ *            argument of the same name of aaac_fit_layer_sel; every layer has its own ws
+ *   mode, group, sel_group, n_outer, n_inner, init   shared by all layers of the batch
+ * Returns the first error found (nothing is enqueued for an invalid batch).
+ */
+typedef struct {
+    const void* W;
+    int64_t N, K, ldw;
+    const float* I;          /* [K], or NULL with X given */
+    const void* X;
+    int64_t T, ldx;
+    float* T01;              /* [2][16] in (AAAC_INIT_USER) / out */
+    void* scales;            /* out */
+    float* tensor_scale;     /* out [1] */
+    double* err_trace;       /* out [n_outer] or NULL */
+    void* ws;
+    size_t ws_bytes;
+} aaac_layer;
+
+int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group, int sel_group,
+                    int n_outer, int n_inner, int init, uint32_t* dev_status /* may be NULL */, void* stream);
+
+/*
  * Per-input-channel scaling before the fit (Section 4, "Combining AAAC with AWQ": AWQ scales
  * the weights, AAAC then learns its tables on the scaled distribution).  The multipliers a_k
  * themselves come from the caller (AWQ's search is not part of the method).

@@ -23,11 +23,18 @@ _lib = None
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
-           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait"]
+           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait", "aaac_fit_layers"]
 
 
 class AaacError(RuntimeError):
     pass
+
+
+class LayerDesc(C.Structure):
+    """aaac_layer of include/aaac.h."""
+    _fields_ = [("W", C.c_void_p), ("N", C.c_int64), ("K", C.c_int64), ("ldw", C.c_int64), ("I", C.c_void_p),
+                ("X", C.c_void_p), ("T", C.c_int64), ("ldx", C.c_int64), ("T01", C.c_void_p), ("scales", C.c_void_p),
+                ("tensor_scale", C.c_void_p), ("err_trace", C.c_void_p), ("ws", C.c_void_p), ("ws_bytes", C.c_size_t)]
 
 
 def lib():
@@ -63,6 +70,8 @@ def lib():
         L.aaac_quantize_layer_host_async.argtypes = [vp, i64, i64, ci, ci, vp, i64, ci, ci, vp, vp, vp, vp, vp, vp, vp,
                                                      vp, C.c_size_t, vp]
         L.aaac_quantize_layer_host_async.restype = ci
+        L.aaac_fit_layers.argtypes = [C.POINTER(LayerDesc), ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.aaac_fit_layers.restype = ci
         L.aaac_debug_fit_wait.argtypes = [ci, C.c_uint]
         L.aaac_debug_fit_wait.restype = ci
         L.aaac_launch_count.restype = C.c_ulonglong
@@ -129,6 +138,24 @@ def fit_layer(W, mode, *, I=None, X=None, n_outer, init, T01, scales, tensor_sca
     _check(lib().aaac_fit_layer(_ptr(W), N, K, W.stride(0), mode, group or group_of(mode), _ptr(I), _ptr(X), T, ldx,
                                 n_outer, n_inner, init, _ptr(T01), _ptr(scales), _ptr(tensor_scale), _ptr(err_trace),
                                 _ptr(dev_status), _ptr(ws), ws.numel(), _stream()))
+
+
+def fit_layers(layers, mode, *, n_outer, init, n_inner=1, group=None, sel_group=None, dev_status=None):
+    """aaac_fit_layers: `layers` is a list of dicts with the keyword arguments of fit_layer that belong
+    to one layer (W, I or X, T01, scales, tensor_scale, ws, optionally err_trace)."""
+    g = group or group_of(mode)
+    arr = (LayerDesc * len(layers))()
+    for d, a in zip(arr, layers):
+        W, X = a["W"], a.get("X")
+        d.W, d.N, d.K, d.ldw = W.data_ptr(), W.shape[0], W.shape[1], W.stride(0)
+        d.I = a["I"].data_ptr() if a.get("I") is not None else None
+        d.X = X.data_ptr() if X is not None else None
+        d.T, d.ldx = (X.shape[0], X.stride(0)) if X is not None else (0, 0)
+        d.T01, d.scales, d.tensor_scale = a["T01"].data_ptr(), a["scales"].data_ptr(), a["tensor_scale"].data_ptr()
+        d.err_trace = a["err_trace"].data_ptr() if a.get("err_trace") is not None else None
+        d.ws, d.ws_bytes = a["ws"].data_ptr(), a["ws"].numel()
+    _check(lib().aaac_fit_layers(arr, len(layers), mode, g, sel_group or g, n_outer, n_inner, init, _ptr(dev_status),
+                                 _stream()))
 
 
 def pack(W, mode, *, I, T01, T01_bf16, scales, tensor_scale, codes, ws, err_out=None, stats=None, group=None,

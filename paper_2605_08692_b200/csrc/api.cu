@@ -135,39 +135,62 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
                               tensor_scale, err_trace, dev_status, ws, ws_bytes, stream);
 }
 
-int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
-                       const float* I, const void* X, int64_t T, int64_t ldx,
-                       int n_outer, int n_inner, int init,
-                       float* T01, void* scales, float* tensor_scale, double* err_trace,
-                       uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
-    int rc = check_layer(W, N, K, ldw, mode, group);
+namespace {
+// argument checks of one layer of a fit call
+int check_fit_layer(const aaac_layer& L, int mode, int group, int sel_group, int n_outer, int n_inner, int init) {
+    int rc = check_layer(L.W, L.N, L.K, L.ldw, mode, group);
     if (rc) return rc;
     if (!sel_ok(mode, group, sel_group)) return AAAC_ERR_MODE;
-    if (!T01 || !scales || !tensor_scale) return AAAC_ERR_NULL;
-    if (!I && !X) return AAAC_ERR_NULL;
+    if (!L.T01 || !L.scales || !L.tensor_scale) return AAAC_ERR_NULL;
+    if (!L.I && !L.X) return AAAC_ERR_NULL;
     if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID && init != AAAC_INIT_USER) return AAAC_ERR_MODE;
     if (n_outer < 0) return AAAC_ERR_SHAPE;
     if (n_inner < 1 || (int64_t)n_outer * n_inner > (1 << 20)) return AAAC_ERR_SHAPE;
-    if (!I && (T < 1 || ldx < K || ldx % 8)) return AAAC_ERR_SHAPE;
-    if (!I && !aligned(X, 16)) return AAAC_ERR_ALIGN;
-    if (I && !aligned(I, 16)) return AAAC_ERR_ALIGN;
-    if (!aligned(scales, mode == AAAC_INT4 ? 2 : 1) || !aligned(T01, 4)) return AAAC_ERR_ALIGN;
-    rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
-    if (rc) return rc;
-    Workspace w = carve(ws, mode, N, K);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const uint16_t* Wp = static_cast<const uint16_t*>(W);
+    if (!L.I && (L.T < 1 || L.ldx < L.K || L.ldx % 8)) return AAAC_ERR_SHAPE;
+    if (!L.I && !aligned(L.X, 16)) return AAAC_ERR_ALIGN;
+    if (L.I && !aligned(L.I, 16)) return AAAC_ERR_ALIGN;
+    if (!aligned(L.scales, mode == AAAC_INT4 ? 2 : 1) || !aligned(L.T01, 4)) return AAAC_ERR_ALIGN;
+    return check_ws(L.ws, L.ws_bytes, carve(nullptr, mode, L.N, L.K).bytes);
+}
 
+// Alg. 1 lines 1-5 of one layer: importance (if from X), scales, start tables; returns the importance used
+int prepare_fit_layer(const aaac_layer& L, int mode, int init, uint32_t* dev_status, const Workspace& w, cudaStream_t st,
+                      const float** I_used) {
+    const uint16_t* Wp = static_cast<const uint16_t*>(L.W);
     if (cudaMemsetAsync(w.ctrl, 0, sizeof(Ctrl), st) != cudaSuccess) return AAAC_ERR_CUDA;
+    const float* I = L.I;
     if (!I) {
-        if (launch_act_stats(static_cast<const uint16_t*>(X), T, K, ldx, w.I, 0, dev_status, w, st) != cudaSuccess)
+        if (launch_act_stats(static_cast<const uint16_t*>(L.X), L.T, L.K, L.ldx, w.I, 0, dev_status, w, st) != cudaSuccess)
             return AAAC_ERR_CUDA;
         I = w.I;
     }
-    if (launch_scales(Wp, N, K, ldw, mode, scales, tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
-    if (launch_init(Wp, N, K, ldw, mode, init, scales, T01, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
-    {
-        // all rounds run in one launch; the optional timing brackets that launch
+    if (launch_scales(Wp, L.N, L.K, L.ldw, mode, L.scales, L.tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (launch_init(Wp, L.N, L.K, L.ldw, mode, init, L.scales, L.T01, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    *I_used = I;
+    return AAAC_OK;
+}
+}  // namespace
+
+int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group, int sel_group,
+                    int n_outer, int n_inner, int init, uint32_t* dev_status, void* stream) {
+    if (!layers) return AAAC_ERR_NULL;
+    if (n_layers < 1 || n_layers > 4096) return AAAC_ERR_SHAPE;
+    for (int l = 0; l < n_layers; ++l) {
+        const int rc = check_fit_layer(layers[l], mode, group, sel_group, n_outer, n_inner, init);
+        if (rc) return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    FitLayerArgs* args = new FitLayerArgs[(size_t)n_layers];
+    int rc = AAAC_OK;
+    for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
+        const aaac_layer& L = layers[l];
+        const Workspace w = carve(L.ws, mode, L.N, L.K);
+        const float* I = nullptr;
+        rc = prepare_fit_layer(L, mode, init, dev_status, w, st, &I);
+        args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, w};
+    }
+    if (rc == AAAC_OK) {
+        // all rounds run in one launch per batch; the optional timing brackets the launches of this call
         cudaEvent_t e0 = nullptr, e1 = nullptr;
         if (n_outer > 0) {
             std::lock_guard<std::mutex> lk(g_timing.mu);
@@ -178,11 +201,22 @@ int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mod
             }
         }
         if (e0) cudaEventRecord(e0, st);
-        if (launch_fit_rounds(Wp, N, K, ldw, mode, sel_group, scales, I, n_outer, n_inner, err_trace, dev_status, w, st) != cudaSuccess)
-            return AAAC_ERR_CUDA;
+        if (launch_fit_rounds_batch(args, n_layers, mode, sel_group, n_outer, n_inner, dev_status, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
         if (e1) cudaEventRecord(e1, st);
     }
-    return launch_export_tables(T01, w, st) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+    for (int l = 0; l < n_layers && rc == AAAC_OK; ++l)
+        if (launch_export_tables(layers[l].T01, args[l].ws, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
+    delete[] args;
+    return rc;
+}
+
+int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group, int sel_group,
+                       const float* I, const void* X, int64_t T, int64_t ldx,
+                       int n_outer, int n_inner, int init,
+                       float* T01, void* scales, float* tensor_scale, double* err_trace,
+                       uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+    const aaac_layer L{W, N, K, ldw, I, X, T, ldx, T01, scales, tensor_scale, err_trace, ws, ws_bytes};
+    return aaac_fit_layers(&L, 1, mode, group, sel_group, n_outer, n_inner, init, dev_status, stream);
 }
 
 int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,

@@ -158,10 +158,17 @@ enum PassKind { kRounds = 0, kAssignKeep = 1, kInner = 2 };
 // to the calling lane's bins under the chosen table, with the arithmetic of the row pipeline
 // (centred term I (x - c), c the chosen entry's centre constant).  Every lane of the warp calls;
 // returns the sum of the groups' smaller errors in lane 0 (0 elsewhere).
+struct DeferArgs {                // what the routine needs of the layer (passed by value: the kernel's
+    const uint16_t* W;            // parameters themselves stay where they are)
+    int64_t K, ldw;
+    const uint8_t* scales;
+    const float* rinv;
+    const float* I;
+    uint32_t* sigw;
+};
 template <int MODE, int SEL, int KIND>
-__device__ __noinline__ double resolve_deferred(const FitTables* S, const FitParams* pp, uint32_t list_addr, int count,
+__device__ __noinline__ double resolve_deferred(const FitTables* S, const DeferArgs p, uint32_t list_addr, int count,
                                                 uint32_t bins_lane, int lane) {
-    const FitParams& p = *pp;
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
     constexpr int WPL = SEL >= 32 ? SEL / 32 : 1;        // weights per lane
     constexpr int ACTIVE = SEL / WPL;                    // lanes that hold weights of the group (32 or 16)
@@ -233,8 +240,10 @@ __device__ __noinline__ double resolve_deferred(const FitTables* S, const FitPar
 
 // SEL is the selection group size S (Sec. 3.1): the weights that share one codebook choice; the
 // scale group g is fixed by the format.
+// The passes of one layer, run by the nblk blocks bid = 0 .. nblk - 1 (a whole grid, or the part
+// of a grid that a batch of layers gives to this layer).
 template <int MODE, int SEL, int NW, int REP, int KIND>
-__global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
+__device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsigned bid, const unsigned nblk) {
     constexpr int NB = AAAC_FIT_BINS;
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
     constexpr int LPG = SEL / 8;                         // lanes per selection group
@@ -266,10 +275,10 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     // A block takes a contiguous range of whole items; what does not divide evenly (the items from
     // tail_item0 on) is dealt out one quarter item -- one row per warp -- per block, so that the
     // busiest block has at most a quarter item more than the others.
-    const int it0 = blockIdx.x * p.per_block;
+    const int it0 = (int)bid * p.per_block;
     const int it1 = min(p.tail_item0, it0 + p.per_block);
-    const bool has_tail = (int)blockIdx.x < p.tail_quarters;
-    const int tail_item = p.tail_item0 + ((int)blockIdx.x >> 2), tail_u = (int)blockIdx.x & 3;
+    const bool has_tail = (int)bid < p.tail_quarters;
+    const int tail_item = p.tail_item0 + ((int)bid >> 2), tail_u = (int)bid & 3;
     static_assert(R == 4, "a tail quarter is one of the four rows of a warp");
 
     if (tid < 2 * kM) S.Td[tid] = p.ctrl->T[tid];
@@ -314,7 +323,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
     // block 0 clears the buffer of the next pass: it was the buffer of two passes ago, and every block
     // finished reading it before it added to the previous pass's buffer, whose totals block 0 has seen
     static_assert(NT >= 256 + kUsed * kLimbs, "threads 256.. of block 0 clear the next buffer");
-    if (blockIdx.x == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs) {
+    if (bid == 0 && tid >= 256 && tid < 256 + kUsed * kLimbs) {
         p.acc[(size_t)((pass_no + 1u) % 3u) * kAccBuffer + (size_t)(tid - 256) * kAccStride] = 0ull;
         __threadfence();
     }
@@ -564,13 +573,13 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         Eacc += (double)eitem;
         if (!INNER && ndefer > kDeferCap - R * (32 / LPG)) {    // the next item could overflow the list
             __syncwarp();
-            Eacc += resolve_deferred<MODE, SEL, KIND>(&S, &p, list_addr, ndefer, bins_lane, lane);
+            Eacc += resolve_deferred<MODE, SEL, KIND>(&S, DeferArgs{p.W, p.K, p.ldw, p.scales, p.rinv, p.I, p.sigw}, list_addr, ndefer, bins_lane, lane);
             ndefer = 0;
         }
     }
     if (!INNER && ndefer > 0) {
         __syncwarp();
-        Eacc += resolve_deferred<MODE, SEL, KIND>(&S, &p, list_addr, ndefer, bins_lane, lane);
+        Eacc += resolve_deferred<MODE, SEL, KIND>(&S, DeferArgs{p.W, p.K, p.ldw, p.scales, p.rinv, p.I, p.sigw}, list_addr, ndefer, bins_lane, lane);
     }
    };
     pass(std::integral_constant<bool, KIND == kInner>{});
@@ -649,7 +658,7 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
             if (spins >= p.spin_limit || ld_relaxed_u32(&p.ctrl->abort)) { ok = false; break; }
             __nanosleep(64);
         }
-        const long long l2 = (long long)(w2 & kLimbMask) - (long long)gridDim.x * kTopBias;
+        const long long l2 = (long long)(w2 & kLimbMask) - (long long)nblk * kTopBias;
         __int128 v = ((__int128)l2 << 64) + ((__int128)(w1 & kLimbMask) << 32) + (__int128)(w0 & kLimbMask);
         const bool neg = v < 0;
         if (neg) v = -v;
@@ -680,11 +689,41 @@ __global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams 
         S.Td[(tid & 16) + rank] = t;
     }
     // the trace holds the Eq. 8 objective of each assignment step
-    if (KIND != kInner && blockIdx.x == 0 && tid == 0 && p.err_trace)
+    if (KIND != kInner && bid == 0 && tid == 0 && p.err_trace)
         p.err_trace[p.trace_base + round] = S.tot[2 * kCells];
     __syncthreads();
   }
-    if (blockIdx.x == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
+    if (bid == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
+}
+
+template <int MODE, int SEL, int NW, int REP, int KIND>
+__global__ void __launch_bounds__(NW * 32, 1) fit_rounds_kernel(const FitParams p) {
+    fit_rounds_body<MODE, SEL, NW, REP, KIND>(p, blockIdx.x, gridDim.x);
+}
+
+// Several layers in one launch (the paper processes layers independently, Sec. 3.3): the grid is
+// cut into consecutive ranges of blocks, one per layer, and every range runs that layer's rounds
+// by itself -- its blocks wait only for each other, on the layer's own accumulators -- so the
+// per-round fixed cost (sums across blocks, new tables, table building) is paid once for the
+// whole batch instead of once per layer, and small layers no longer leave most of the GPU idle.
+// The parameters of every layer stay kernel arguments (one copy of the code per slot).
+constexpr int kMaxBatch = 8;
+struct FitBatch {
+    FitParams L[kMaxBatch];
+    unsigned first[kMaxBatch + 1];    // first block of every layer; first[n..] = grid size
+};
+
+template <int MODE, int SEL, int NW, int REP>
+__global__ void __launch_bounds__(NW * 32, 1) fit_batch_kernel(const FitBatch b) {
+    const unsigned bx = blockIdx.x;
+#define AAAC_BATCH_SLOT(i)                                                                              \
+    if (bx < b.first[i + 1]) {                                                                           \
+        fit_rounds_body<MODE, SEL, NW, REP, kRounds>(b.L[i], bx - b.first[i], b.first[i + 1] - b.first[i]); \
+        return;                                                                                          \
+    }
+    AAAC_BATCH_SLOT(0) AAAC_BATCH_SLOT(1) AAAC_BATCH_SLOT(2) AAAC_BATCH_SLOT(3)
+    AAAC_BATCH_SLOT(4) AAAC_BATCH_SLOT(5) AAAC_BATCH_SLOT(6) AAAC_BATCH_SLOT(7)
+#undef AAAC_BATCH_SLOT
 }
 
 __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
@@ -705,23 +744,14 @@ cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
 
 }  // namespace
 
-cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
-                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
-                              const Workspace& ws, cudaStream_t st) {
-    if (n_outer <= 0) return cudaSuccess;
-    if (n_inner < 1 || (int64_t)n_outer * n_inner > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    FitParams p{};
-    p.W = W; p.N = N; p.K = K; p.ldw = ldw;
-    p.scales = static_cast<const uint8_t*>(scales); p.rinv = ws.rinv; p.I = I;
-    p.ctrl = ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(ws.part); p.err_trace = err_trace; p.dev_status = dev_status;
-    p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
-    p.spin_limit = g_spin_limit;
-    p.sigw = ws.qlist;            // the quantile selection's list is free once the start tables exist
+// Deals a layer's items to `blocks` blocks: whole items in contiguous ranges plus, where that is
+// shorter for the busiest block, a tail dealt out one row per warp (a quarter item) per block.
+// Returns the number of blocks actually used.
+static int64_t plan_layer(FitParams& p, int64_t N, int64_t K, int64_t blocks) {
     const int64_t slabs = (K + 255) / 256;
     constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
     const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
-    if (N > 0x7FFFFFFF || K > 0x7FFFFFFF || items > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    int64_t grid = sm_count();
+    int64_t grid = blocks;
     if (grid > items) grid = items;
     if (grid > kMaxFitBlocks) grid = kMaxFitBlocks;
     int64_t per_block = (items + grid - 1) / grid;
@@ -730,7 +760,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     {
         // an even number of whole items per block plus a quarter-item tail, where that is shorter for
         // the busiest block (a tail row costs more than a quarter of a pipelined item: count it double)
-        const int64_t g = sm_count() < kMaxFitBlocks ? sm_count() : kMaxFitBlocks;
+        const int64_t g = blocks < kMaxFitBlocks ? blocks : kMaxFitBlocks;
         const int64_t whole = items / g, rest = items - whole * g;
         if (whole >= 4 && rest > 0 && 4 * rest <= g && 2 * whole + 1 < 2 * per_block) {
             per_block = whole;
@@ -742,6 +772,32 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
     if (p.tail_quarters == 0) grid = (items + per_block - 1) / per_block;
     p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
     p.arrivals = (unsigned)grid + (unsigned)g_extra_arrivals;
+    return grid;
+}
+
+static bool fill_params(FitParams& p, const FitLayerArgs& a, int n_outer, uint32_t* dev_status) {
+    p = FitParams{};
+    p.W = a.W; p.N = a.N; p.K = a.K; p.ldw = a.ldw;
+    p.scales = static_cast<const uint8_t*>(a.scales); p.rinv = a.ws.rinv; p.I = a.I;
+    p.ctrl = a.ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(a.ws.part); p.err_trace = a.err_trace; p.dev_status = dev_status;
+    p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
+    p.spin_limit = g_spin_limit;
+    p.sigw = a.ws.qlist;            // the quantile selection's list is free once the start tables exist
+    const int64_t slabs = (a.K + 255) / 256;
+    constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
+    const int64_t nrb = (a.N + kRowsPerItem - 1) / kRowsPerItem;
+    return !(a.N > 0x7FFFFFFF || a.K > 0x7FFFFFFF || slabs * nrb > 0x7FFFFFFF);
+}
+
+cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
+                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
+                              const Workspace& ws, cudaStream_t st) {
+    if (n_outer <= 0) return cudaSuccess;
+    if (n_inner < 1 || (int64_t)n_outer * n_inner > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    FitLayerArgs a{W, N, K, ldw, scales, I, err_trace, ws};
+    FitParams p;
+    if (!fill_params(p, a, n_outer, dev_status)) return cudaErrorInvalidValue;
+    const int64_t grid = plan_layer(p, N, K, sm_count());
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
     auto launch = [&](auto kind) {
         constexpr int KIND = decltype(kind)::value;
@@ -763,6 +819,74 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
         e = launch(std::integral_constant<int, kInner>{});
         if (e != cudaSuccess) return e;
         p.bar_base += (unsigned)(n_inner - 1);
+    }
+    return cudaSuccess;
+}
+
+template <int MODE, int SEL>
+static cudaError_t launch_batch_variant(FitBatch& b, unsigned grid, cudaStream_t st) {
+    constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
+    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kLut2Bytes + (size_t)NW * kBinSlots * kSlotBytes + (size_t)NW * kDeferCap * 8;
+    auto kern = fit_batch_kernel<MODE, SEL, NW, REP>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    void* args[] = {&b};
+    note_launch();
+    // cooperative: the blocks of a layer wait for each other, so all of them must be resident
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kern), dim3(grid), dim3(NW * 32), args, smem, st);
+}
+
+cudaError_t launch_fit_rounds_batch(const FitLayerArgs* layers, int n, int mode, int sel_group, int n_outer, int n_inner,
+                                    uint32_t* dev_status, cudaStream_t st) {
+    if (n_outer <= 0 || n <= 0) return cudaSuccess;
+    if (n_inner < 1 || (int64_t)n_outer * n_inner > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    const int sms = sm_count();
+    for (int at = 0; at < n;) {
+        const int m = (n - at) < kMaxBatch ? (n - at) : kMaxBatch;
+        if (m == 1 || n_inner > 1 || m > sms) {
+            // single layers and inner refinement go through the one-layer launches
+            const FitLayerArgs& a = layers[at];
+            cudaError_t e = launch_fit_rounds(a.W, a.N, a.K, a.ldw, mode, sel_group, a.scales, a.I, n_outer, n_inner,
+                                              a.err_trace, dev_status, a.ws, st);
+            if (e != cudaSuccess) return e;
+            at += 1;
+            continue;
+        }
+        FitBatch b{};
+        int64_t items[kMaxBatch], share[kMaxBatch];
+        constexpr int kRowsPerItem = kRowsPerWarp * AAAC_FIT_WARPS;
+        for (int l = 0; l < m; ++l) {
+            const FitLayerArgs& a = layers[at + l];
+            if (!fill_params(b.L[l], a, n_outer, dev_status)) return cudaErrorInvalidValue;
+            items[l] = ((a.K + 255) / 256) * ((a.N + kRowsPerItem - 1) / kRowsPerItem);
+            share[l] = 1;
+        }
+        // one block per layer, then every further block to the layer whose busiest block has the most items
+        for (int left = sms - m; left > 0; --left) {
+            int best = -1;
+            int64_t load = 0;
+            for (int l = 0; l < m; ++l) {
+                const int64_t per = (items[l] + share[l] - 1) / share[l];
+                if (share[l] < items[l] && share[l] < kMaxFitBlocks && per > load) { load = per; best = l; }
+            }
+            if (best < 0) break;
+            ++share[best];
+        }
+        unsigned grid = 0;
+        for (int l = 0; l < m; ++l) {
+            const FitLayerArgs& a = layers[at + l];
+            b.first[l] = grid;
+            grid += (unsigned)plan_layer(b.L[l], a.N, a.K, share[l]);
+            cudaError_t em = cudaMemsetAsync(b.L[l].acc, 0, sizeof(unsigned long long) * 3 * kAccBuffer, st);
+            if (em != cudaSuccess) return em;
+        }
+        for (int l = m; l <= kMaxBatch; ++l) b.first[l] = grid;
+        cudaError_t e;
+        if (mode == AAAC_INT4 && sel_group == 16) e = launch_batch_variant<AAAC_INT4, 16>(b, grid, st);
+        else if (mode == AAAC_INT4) e = launch_batch_variant<AAAC_INT4, 128>(b, grid, st);
+        else e = launch_batch_variant<AAAC_NVFP4, 16>(b, grid, st);
+        if (e != cudaSuccess) return e;
+        at += m;
     }
     return cudaSuccess;
 }

@@ -116,6 +116,17 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
                               const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st);
+// the same for several layers of one mode in a single launch (n_inner = 1; otherwise layer by layer)
+struct FitLayerArgs {
+    const uint16_t* W;
+    int64_t N, K, ldw;
+    const void* scales;
+    const float* I;
+    double* err_trace;
+    Workspace ws;
+};
+cudaError_t launch_fit_rounds_batch(const FitLayerArgs* layers, int n, int mode, int sel_group, int n_outer, int n_inner,
+                                    uint32_t* dev_status, cudaStream_t st);
 cudaError_t launch_export_tables(float* T01, const Workspace& ws, cudaStream_t st);
 // sigma_bits: null when the selection group is the scale group (sigma in the scale's sign bit)
 cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const float* I,

@@ -375,6 +375,119 @@ def test_fit_wait_runs_out_and_is_reported():
         assert torch.equal(again[k], good[k]), k
 
 
+# ------------------------------------------------------------------ several layers in one call
+
+def run_fit_batch(cases, mode, rounds, init, n_inner=1, sel_group=None):
+    """aaac_fit_layers on a list of (W, I) cases; returns per layer the fitted tables, scales, trace."""
+    g = 128 if mode == INT4 else 16
+    descs, keep = [], []
+    for W, I in cases:
+        N, K = W.shape
+        d = dict(W=dev_bf16(W), I=torch.from_numpy(np.ascontiguousarray(I)).to(DEV),
+                 T01=torch.zeros(2, 16, dtype=torch.float32, device=DEV),
+                 scales=torch.empty(N, K // g, dtype=torch.uint16 if mode == INT4 else torch.uint8, device=DEV),
+                 tensor_scale=torch.ones(1, dtype=torch.float32, device=DEV),
+                 err_trace=torch.zeros(max(rounds, 1), dtype=torch.float64, device=DEV),
+                 ws=binding.alloc_workspace(mode, N, K))
+        descs.append(d)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.fit_layers(descs, mode, n_outer=rounds, init=init, n_inner=n_inner, sel_group=sel_group, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return descs
+
+
+@pytest.mark.parametrize("mode", [INT4, NVFP4])
+def test_fit_layers_batch_matches_oracle_per_layer(mode):
+    """Several layers of different shapes (ragged rows and columns, a one-row layer) fitted in one
+    call: every layer against the oracle, like a layer fitted alone; twice for reproducibility."""
+    g = 128 if mode == INT4 else 16
+    shapes = [(257, 1024), (3, 256), (70, 640), (1, 128), (300, 768)]
+    cases, oracles = [], []
+    for i, (N, K) in enumerate(shapes):
+        W, X = layer(mode, N, K, name=f"batch{mode}/{i}")
+        o = oracle.fit_layer(W, mode, g, 6, X=X, init="quantile")
+        cases.append((W, o["I"]))
+        oracles.append(o)
+    a = run_fit_batch(cases, mode, 6, binding.INIT_QUANTILE)
+    b = run_fit_batch(cases, mode, 6, binding.INIT_QUANTILE)
+    for i, (d, d2, o) in enumerate(zip(a, b, oracles)):
+        ok, worst = table_close(host(d["T01"]), o["T"])
+        assert ok, f"layer {i}: tables differ: worst {worst:.3e}"
+        tr = host(d["err_trace"])[:6]
+        assert np.allclose(tr, o["trace"], rtol=1e-4, atol=0)
+        assert np.array_equal(host(d["scales"]), o["scales_unsigned"])
+        assert torch.equal(d["T01"], d2["T01"]) and torch.equal(d["err_trace"], d2["err_trace"])
+        # and the pack pass from these tables gives the oracle's bits
+        W = cases[i][0]
+        r = dict(T01_bf16=None)
+        Tb = torch.empty(2, 16, dtype=torch.uint16, device=DEV)
+        codes = torch.empty(W.shape[0], W.shape[1] // 2, dtype=torch.uint8, device=DEV)
+        binding.pack(d["W"], mode, I=d["I"], T01=d["T01"], T01_bf16=Tb, scales=d["scales"], tensor_scale=d["tensor_scale"],
+                     codes=codes, ws=d["ws"])
+        assert np.array_equal(host(Tb), o["T_bf16"]), f"layer {i}: BF16 tables differ"
+        assert np.array_equal(host(codes), o["codes"]) and np.array_equal(host(d["scales"]), o["scales"])
+
+
+def test_fit_layers_more_layers_than_one_launch_takes_and_inner_refinement():
+    """Eleven layers (more than one launch holds) and a batch with n_inner > 1 (run layer by layer)."""
+    rng = np.random.default_rng(3)
+    cases, oracles = [], []
+    for i in range(11):
+        N, K = int(rng.integers(1, 90)), 256 * int(rng.integers(1, 4))
+        W, X = layer(NVFP4, N, K, name=f"batch11/{i}")
+        o = oracle.fit_layer(W, NVFP4, 16, 3, X=X, init="grid")
+        cases.append((W, o["I"]))
+        oracles.append(o)
+    for d, o in zip(run_fit_batch(cases, NVFP4, 3, binding.INIT_GRID), oracles):
+        assert table_close(host(d["T01"]), o["T"])[0]
+    cases, oracles = [], []
+    for i, (N, K) in enumerate([(70, 640), (130, 512)]):
+        W, X = layer(INT4, N, K, name=f"batchinner/{i}")
+        o = oracle.fit_layer(W, INT4, 128, 2, X=X, init="quantile", n_inner=3, S=16)
+        cases.append((W, o["I"]))
+        oracles.append(o)
+    for d, o in zip(run_fit_batch(cases, INT4, 2, binding.INIT_QUANTILE, n_inner=3, sel_group=16), oracles):
+        assert table_close(host(d["T01"]), o["T"])[0]
+        assert np.allclose(host(d["err_trace"])[:2], o["trace"], rtol=1e-4)
+
+
+def test_fit_layers_rejects_a_bad_layer_before_enqueuing_anything():
+    W, X = layer(NVFP4, 16, 256, name="batchbad")
+    good = dict(W=dev_bf16(W), I=torch.ones(256, device=DEV), T01=torch.zeros(2, 16, device=DEV),
+                scales=torch.empty(16, 16, dtype=torch.uint8, device=DEV), tensor_scale=torch.ones(1, device=DEV),
+                ws=binding.alloc_workspace(NVFP4, 16, 256))
+    bad = dict(good, ws=torch.empty(64, dtype=torch.uint8, device=DEV))       # workspace too small
+    before = binding.launch_count()
+    with pytest.raises(binding.AaacError, match="status 5"):
+        binding.fit_layers([good, bad], NVFP4, n_outer=2, init=binding.INIT_GRID)
+    assert binding.launch_count() == before
+
+
+def test_config2_layers_in_one_batch_full_size():
+    """The benchmark's three layers fitted in one call (the launch configuration the benchmark times):
+    each against the whole-layer oracle."""
+    cases, oracles = [], []
+    for which in ("q_proj", "gate_proj", "down_proj"):
+        c = synth.config2_layer(which)
+        o = oracle.fit_layer(c["W"], NVFP4, 16, c["rounds"], X=c["X"], init="quantile")
+        cases.append((c["W"], o["I"]))
+        oracles.append(o)
+    for which, d, o in zip(("q_proj", "gate_proj", "down_proj"), run_fit_batch(cases, NVFP4, 20, binding.INIT_QUANTILE), oracles):
+        ok, worst = table_close(host(d["T01"]), o["T"])
+        assert ok, f"{which}: tables differ: worst {worst:.3e}"
+        tr = host(d["err_trace"])[:20]
+        assert np.allclose(tr, o["trace"], rtol=1e-4, atol=0) and np.all(tr[1:] <= tr[:-1] * (1 + 1e-6))
+        Tb = torch.empty(2, 16, dtype=torch.uint16, device=DEV)
+        codes = torch.empty(d["W"].shape[0], d["W"].shape[1] // 2, dtype=torch.uint8, device=DEV)
+        binding.pack(d["W"], NVFP4, I=d["I"], T01=d["T01"], T01_bf16=Tb, scales=d["scales"], tensor_scale=d["tensor_scale"],
+                     codes=codes, ws=d["ws"])
+        differ = int(np.sum(host(Tb) != o["T_bf16"]))
+        print(f"batched {which}: worst table deviation {worst:.2e}, BF16 entries that differ {differ}")
+        assert differ == 0
+        assert np.array_equal(host(codes), o["codes"]) and np.array_equal(host(d["scales"]), o["scales"])
+
+
 # ------------------------------------------------------------------ inner refinement (n_inner > 1)
 
 @pytest.mark.parametrize("mode,init", [(INT4, "grid"), (INT4, "quantile"), (NVFP4, "quantile")])
