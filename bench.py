@@ -316,6 +316,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-seconds", type=float, default=120.0,
                     help="reference arm: CPU seconds the whole run should take (bounds the sample per step)")
+    ap.add_argument("--with-prescale", action="store_true",
+                    help="profiling runs: also scale every layer's input channels (aaac_prescale_columns, unit "
+                         "multipliers) at the start of a step, so that the kernel shows up in a capture")
     ap.add_argument("--no-stacks", action="store_true",
                     help="leave the decoder-stack wall times out of the line (profiling runs)")
     ap.add_argument("--layers", default=",".join(LAYERS),
@@ -391,12 +394,16 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
     descs = [dict(W=W, I=o["I"], T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"]) for W, o in zip(Wd, outs)]
+    ones = {K: torch.ones(K, dtype=torch.float32, device=dev) for _, K in shapes} if args.with_prescale else {}
 
     def step():
         # the layers of a step are independent: their importances first, then scales, start tables and the
         # 20 rounds of all of them in one aaac_fit_layers call (the rounds in one launch), then pack and dequant
         for X, o in zip(Xd, outs):
             binding.act_stats(X, o["I"], o["ws"], dev_status=status)
+        if args.with_prescale:
+            for W, o in zip(Wd, outs):
+                binding.prescale_columns(W, ones[W.shape[1]], o["What"], o["I"], o["I"], dev_status=status)
         binding.fit_layers(descs, mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE, dev_status=status)
         for W, o in zip(Wd, outs):
             binding.pack(W, mode, I=o["I"], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"], tensor_scale=o["ts"],

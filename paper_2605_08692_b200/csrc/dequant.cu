@@ -61,9 +61,10 @@ dequant_kernel(const uint8_t* __restrict__ codes, const void* __restrict__ scale
             uint32_t o[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t lo = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j)) & 15u], s));
-                const uint32_t hi = f32_to_bf16_rne(__fmul_rn(Ts[(word >> (8 * j + 4)) & 15u], s));
-                o[j] = lo | (hi << 16);
+                // two products rounded to BF16 (nearest even) and packed by one conversion instruction
+                const float lo = __fmul_rn(Ts[(word >> (8 * j)) & 15u], s);
+                const float hi = __fmul_rn(Ts[(word >> (8 * j + 4)) & 15u], s);
+                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[j]) : "f"(hi), "f"(lo));
             }
             __stcs(reinterpret_cast<uint4*>(What + row * ldo + col), make_uint4(o[0], o[1], o[2], o[3]));
         }

@@ -31,9 +31,11 @@ __device__ __forceinline__ uint32_t float_key(float f) {      // order-preservin
 __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
+// bin = floor(1024 x + 8192): one multiply-add rounded down onto 1.5 * 2^23 (where floats are
+// spaced by 1) leaves the integer in the low mantissa bits; the mask keeps any input inside the
+// table (|w~| < 8 by the scale rules, so for finite weights it changes nothing)
 __device__ __forceinline__ int qbin(float x) {
-    int b = __float2int_rd(__fmaf_rn(x, 1024.f, 8192.f));
-    return min(max(b, 0), kQBins - 1);
+    return (int)(__float_as_uint(__fmaf_rd(x, 1024.f, 8192.f + 12582912.f)) & (uint32_t)(kQBins - 1));
 }
 
 // reciprocal of the group's scale for the 8 weights a lane holds
@@ -184,18 +186,38 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     flush();
 }
 
-// one block of 1024 threads: prefix sum, bin + local rank of every request, slots
+// one block of 1024 threads: prefix sum, bin + local rank of every request, slots.  Every thread
+// keeps its chunk of 16 bins in registers; the thread whose chunk holds a requested rank walks
+// those registers (no dependent memory reads), and the bin -> slot table is cleared by word stores.
 __global__ void __launch_bounds__(1024)
-quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned long long* __restrict__ prefix,
-                     uint8_t* __restrict__ slot_of_bin) {
+quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __restrict__ slot_of_bin) {
     __shared__ unsigned long long chunk[1024];
+    __shared__ unsigned long long req_rank[kQReq];
     __shared__ int req_bin[kQReq];
+    __shared__ unsigned long long req_cnt[kQReq];
+    __shared__ int req_first[kQReq];
+    __shared__ unsigned long long wtot[32];
     const int tid = threadIdx.x;
     constexpr int per = kQBins / 1024;
+    static_assert(per == 16, "a thread's chunk is four 16-byte loads");
+    uint32_t h[per];
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(hist + tid * per);
+#pragma unroll
+        for (int i = 0; i < per / 4; ++i) {
+            const uint4 v = __ldg(src + i);
+            h[4 * i] = v.x; h[4 * i + 1] = v.y; h[4 * i + 2] = v.z; h[4 * i + 3] = v.w;
+        }
+    }
     unsigned long long s = 0;
-    for (int i = 0; i < per; ++i) s += hist[tid * per + i];
-    chunk[tid] = s;
-    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < per; ++i) s += h[i];
+    if (tid < kQReq) req_rank[tid] = ctrl->rank[tid];
+    {
+        uint32_t* clr = reinterpret_cast<uint32_t*>(slot_of_bin);
+#pragma unroll
+        for (int i = 0; i < kQBins / 4 / 1024; ++i) clr[tid + i * 1024] = 0xFFFFFFFFu;
+    }
     // exclusive prefix of the 1024 chunk sums: warp scans, then a scan of the 32 warp totals
     {
         const int lane = tid & 31, warp = tid >> 5;
@@ -205,7 +227,6 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned lon
             const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, v, o);
             if (lane >= o) v += t;
         }
-        __shared__ unsigned long long wtot[32];
         if (lane == 31) wtot[warp] = v;
         __syncthreads();
         if (warp == 0) {
@@ -221,32 +242,26 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, unsigned lon
         chunk[tid] = v - s + (warp ? wtot[warp - 1] : 0ull);
     }
     __syncthreads();
-    unsigned long long run = chunk[tid];
-    for (int i = 0; i < per; ++i) {
-        prefix[tid * per + i] = run;                      // exclusive prefix
-        run += hist[tid * per + i];
-        slot_of_bin[tid * per + i] = 0xFF;
-    }
-    if (tid == 1023) prefix[kQBins] = run;
-    __syncthreads();
-    __shared__ unsigned long long req_cnt[kQReq];
-    __shared__ int req_first[kQReq];
-    if (tid < kQReq) {
-        // the bin that holds rank r: first the chunk (exclusive chunk prefixes are in shared
-        // memory), then a walk over the chunk's bins
-        const unsigned long long r = ctrl->rank[tid];
-        int lo = 0, hi = 1024;                            // last chunk with chunk[c] <= r
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (chunk[mid] <= r) lo = mid; else hi = mid;
+    {
+        // the requests whose rank lies in this thread's chunk (the last chunk also takes ranks beyond
+        // the data, which are never requested): walk the chunk's bins in registers
+        const unsigned long long lo = chunk[tid], hi = lo + s;
+        for (int q = 0; q < kQReq; ++q) {
+            const unsigned long long r = req_rank[q];
+            if (!(r >= lo && (r < hi || tid == 1023))) continue;
+            if (r >= hi && tid != 1023) continue;
+            unsigned long long base = lo;
+            int i = 0;
+#pragma unroll
+            for (int k = 0; k < per - 1; ++k)
+                if (i == k && r >= base + h[k]) { base += h[k]; ++i; }
+            uint32_t hv = h[0];
+#pragma unroll
+            for (int k = 1; k < per; ++k) if (i == k) hv = h[k];
+            req_bin[q] = tid * per + i;
+            req_cnt[q] = hv;
+            ctrl->req_local[q] = r - base;
         }
-        unsigned long long base = chunk[lo];
-        int b = lo * per;
-        unsigned long long h = hist[b];
-        while (b < kQBins - 1 && r >= base + h) { base += h; ++b; h = hist[b]; }
-        req_bin[tid] = b;
-        req_cnt[tid] = h;
-        ctrl->req_local[tid] = r - base;
     }
     __syncthreads();
     if (tid < kQReq) {
@@ -515,7 +530,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
         quantile_hist_kernel<AAAC_NVFP4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
         note_launch();
     }
-    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qprefix, ws.qslot_of_bin);
+    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qslot_of_bin);
     note_launch();
     const int blocks1 = sm_count() * 4;
     if (mode == AAAC_INT4)
