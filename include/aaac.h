@@ -48,7 +48,7 @@ typedef enum {
     AAAC_ERR_MODE = 2,          /* unknown mode / init, or group does not match the mode */
     AAAC_ERR_SHAPE = 3,         /* N < 1, K % g, K % 8, ld < K, ld % 8, T < 1, n_outer < 0 */
     AAAC_ERR_ALIGN = 4,         /* a pointer is not 16-byte aligned (ws: 256) */
-    AAAC_ERR_WORKSPACE = 5,     /* ws_bytes too small */
+    AAAC_ERR_WORKSPACE = 5,     /* ws_bytes too small (host-buffer calls: also AAAC_DEV_SCRATCH was set) */
     AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
     AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
     AAAC_ERR_UNIMPLEMENTED = 8, /* reserved */
@@ -67,12 +67,23 @@ typedef enum {
 /* bits OR-ed into *dev_status by the kernels */
 #define AAAC_DEV_NONFINITE 1u
 #define AAAC_DEV_TIMEOUT 2u      /* a bounded wait inside a kernel ran out; results are not valid */
+#define AAAC_DEV_SCRATCH 4u      /* the quantile start needed more scratch than ws holds (see aaac_workspace_bytes); the
+                                    start tables, and everything fitted from them, are not valid */
 
 const char* aaac_status_string(int status);
 
 /* Bytes of scratch that any call below needs for a layer of this shape (T = calibration
- * tokens, 0 if activations are never passed). */
+ * tokens, 0 if activations are never passed): a few megabytes of fixed regions plus the candidate
+ * list of the quantile start (Eq. 9-10), 4 bytes for a sixteenth of the layer's weights -- about
+ * an eighth of the layer's own size.  The list holds the normalised weights that fall into the
+ * (at most 64) histogram bins of width 2^-10 around the requested quantiles, usually 1-3 % of
+ * the weights.  A bin whose weights do not fit the list is still resolved when they all have one
+ * value (a constant or pruned layer); otherwise AAAC_DEV_SCRATCH is set in dev_status.  A caller
+ * who wants to rule that out passes a larger workspace: whatever ws_bytes holds beyond the fixed
+ * regions is used for the list, and aaac_workspace_bytes_full is the size that can never fall
+ * short (one list entry per weight: twice the layer's size). */
 size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T);
+size_t aaac_workspace_bytes_full(int mode, int64_t N, int64_t K, int64_t T);
 
 /*
  * Activation importance, Eq. 7:  I[k] = sum_t X[t,k]^2.
@@ -295,6 +306,14 @@ int aaac_timing_end(float* ms_host, int capacity);
  * thread-safe against concurrent aaac_fit_layer calls.
  */
 int aaac_debug_fit_wait(int extra_arrivals, unsigned spin_limit);
+
+/*
+ * Diagnostics for the quantile start's candidate list: entries > 0 caps the list of every later
+ * call of the process at that many entries (never below what the fit's selection words need), so
+ * that the paths taken when a bin's weights do not fit -- one shared value: resolved; several:
+ * AAAC_DEV_SCRATCH -- can be tested on small layers; 0 restores the normal capacity.  Process-wide.
+ */
+int aaac_debug_quantile_cap(size_t entries);
 
 /*
  * Number of kernels this library has launched in the calling process so far (all entry points,

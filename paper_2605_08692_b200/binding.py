@@ -15,6 +15,7 @@ INT4, NVFP4 = 0, 1
 INIT_QUANTILE, INIT_GRID, INIT_USER = 0, 1, 2
 DEV_NONFINITE = 1
 DEV_TIMEOUT = 2          # a bounded wait between the blocks of the fit-rounds kernel ran out: results are not valid
+DEV_SCRATCH = 4          # the quantile start ran out of scratch: pass a larger workspace (workspace_bytes_full)
 ERR_TIMEOUT = 10
 
 _LIB_PATH = os.environ.get("AAAC_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaaac_b200.so")
@@ -23,7 +24,7 @@ _lib = None
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
-           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait", "aaac_fit_layers"]
+           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait", "aaac_fit_layers", "aaac_workspace_bytes_full", "aaac_debug_quantile_cap"]
 
 
 class AaacError(RuntimeError):
@@ -48,6 +49,8 @@ def lib():
         L.aaac_status_string.argtypes = [C.c_int]
         L.aaac_workspace_bytes.restype = C.c_size_t
         L.aaac_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
+        L.aaac_workspace_bytes_full.restype = C.c_size_t
+        L.aaac_workspace_bytes_full.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
         L.aaac_host_workspace_bytes.restype = C.c_size_t
         L.aaac_host_workspace_bytes.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
         vp, i64, ci = C.c_void_p, C.c_int64, C.c_int
@@ -72,6 +75,8 @@ def lib():
         L.aaac_quantize_layer_host_async.restype = ci
         L.aaac_fit_layers.argtypes = [C.POINTER(LayerDesc), ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.aaac_fit_layers.restype = ci
+        L.aaac_debug_quantile_cap.argtypes = [C.c_size_t]
+        L.aaac_debug_quantile_cap.restype = ci
         L.aaac_debug_fit_wait.argtypes = [ci, C.c_uint]
         L.aaac_debug_fit_wait.restype = ci
         L.aaac_launch_count.restype = C.c_ulonglong
@@ -107,8 +112,14 @@ def workspace_bytes(mode: int, N: int, K: int, T: int = 0) -> int:
     return int(lib().aaac_workspace_bytes(mode, N, K, T))
 
 
-def alloc_workspace(mode: int, N: int, K: int, T: int = 0, device="cuda") -> torch.Tensor:
-    return torch.empty(workspace_bytes(mode, N, K, T), dtype=torch.uint8, device=device)
+def workspace_bytes_full(mode: int, N: int, K: int, T: int = 0) -> int:
+    """The workspace size with which the quantile start can never run out of scratch."""
+    return int(lib().aaac_workspace_bytes_full(mode, N, K, T))
+
+
+def alloc_workspace(mode: int, N: int, K: int, T: int = 0, device="cuda", full: bool = False) -> torch.Tensor:
+    nbytes = workspace_bytes_full(mode, N, K, T) if full else workspace_bytes(mode, N, K, T)
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
 
 
 def act_stats(X: torch.Tensor, I: torch.Tensor, ws: torch.Tensor, accumulate: bool = False, dev_status=None):
@@ -220,6 +231,11 @@ def debug_fit_wait(extra_arrivals: int = 0, spin_limit: int = 0):
     """Test hook: make the fit rounds' bounded wait run out (extra_arrivals > 0) after spin_limit
     polls; (0, 0) restores normal operation."""
     _check(lib().aaac_debug_fit_wait(extra_arrivals, spin_limit))
+
+
+def debug_quantile_cap(entries: int = 0):
+    """Test hook: cap the quantile start's candidate list at `entries` (0 restores the normal size)."""
+    _check(lib().aaac_debug_quantile_cap(entries))
 
 
 def launch_count() -> int:

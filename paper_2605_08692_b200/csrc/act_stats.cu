@@ -88,10 +88,17 @@ __global__ void act_final_kernel(const double* __restrict__ part, int splits, in
 
 }  // namespace
 
+int act_splits_max(int64_t K) {
+    const int64_t bx = (K + 255) / 256;
+    int64_t want = ((int64_t)sm_count() * 8 + bx - 1) / (bx > 0 ? bx : 1);
+    if (want < 1) want = 1;
+    return (int)(want > kActMaxSplits ? kActMaxSplits : want);
+}
+
 cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
                              uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
     const int bx = (int)((K + 255) / 256);
-    int64_t want = ((int64_t)sm_count() * 8 + bx - 1) / bx;
+    int64_t want = act_splits_max(K);
     int64_t max_by_rows = (T + kWarps - 1) / kWarps;
     int64_t splits = want < 1 ? 1 : want;
     if (splits > max_by_rows) splits = max_by_rows;

@@ -28,8 +28,24 @@ namespace {
 constexpr size_t kAlign = 256;
 size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Lays the scratch regions out after `base` (which may be null to measure only).
-Workspace carve(void* base, int mode, int64_t N, int64_t K) {
+// Candidate list of the quantile start: by default a sixteenth of the layer's weights (what the
+// <= 64 histogram bins of the requested order statistics hold is usually 1-3 %), never less than
+// the fit's selection words [N][ceil(K/256)] that later reuse the space.
+size_t g_debug_qcap = 0;         // aaac_debug_quantile_cap: a forced list capacity (0 = none)
+
+size_t default_qcap(int64_t N, int64_t K) {
+    if (N <= 0 || K <= 0) return 1;
+    const size_t nk = (size_t)N * (size_t)K;
+    size_t cap = nk / 16;
+    if (cap < ((size_t)1 << 18)) cap = nk < ((size_t)1 << 18) ? nk : ((size_t)1 << 18);
+    const size_t sig = (size_t)N * (size_t)((K + 255) / 256);
+    return cap < sig ? sig : cap;
+}
+
+// Lays the scratch regions out after `base` (which may be null to measure only).  qcap = entries
+// of the candidate list; with a real workspace the list takes whatever the caller's buffer holds
+// beyond the fixed regions (at most one entry per weight).
+Workspace carve(void* base, int mode, int64_t N, int64_t K, size_t ws_bytes = 0, bool full = false) {
     Workspace w{};
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -40,14 +56,23 @@ Workspace carve(void* base, int mode, int64_t N, int64_t K) {
     const int g = mode == AAAC_INT4 ? 128 : 16;
     const int64_t K8 = (K + 7) / 8 * 8;
     w.ctrl = static_cast<Ctrl*>(take(sizeof(Ctrl)));
-    w.part = static_cast<double*>(take(sizeof(double) * 2 * kMaxBlocks * kPartStride));
-    w.rinv = static_cast<float*>(take(sizeof(float) * (size_t)(N > 0 && K > 0 ? N * (K / g + 1) : 1)));
+    w.part = static_cast<double*>(take(sizeof(double) * kMaxBlocks * kPartStride));
+    w.rinv = static_cast<float*>(take(sizeof(float) * (size_t)(mode == AAAC_INT4 && N > 0 && K > 0 ? N * (K / g + 1) : 1)));
     w.I = static_cast<float*>(take(sizeof(float) * (size_t)(K8 > 0 ? K8 : 8)));
-    w.act_part = static_cast<double*>(take(sizeof(double) * kActMaxSplits * (size_t)(K8 > 0 ? K8 : 8)));
+    w.act_part = static_cast<double*>(take(sizeof(double) * (size_t)act_splits_max(K) * (size_t)(K8 > 0 ? K8 : 8)));
     w.qhist = static_cast<uint32_t*>(take(sizeof(uint32_t) * kQBins));
-    w.qprefix = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * (kQBins + 1)));
     w.qslot_of_bin = static_cast<uint8_t*>(take(kQBins));
-    w.qlist = static_cast<uint32_t*>(take(sizeof(uint32_t) * (size_t)(N > 0 && K > 0 ? N * K : 1)));
+    const size_t nk = (size_t)(N > 0 && K > 0 ? N * K : 1);
+    size_t cap = full ? nk : default_qcap(N, K);
+    if (base && ws_bytes > off + cap * sizeof(uint32_t)) {
+        cap = (ws_bytes - off) / sizeof(uint32_t);
+        if (cap > nk) cap = nk;
+    }
+    if (g_debug_qcap && g_debug_qcap < cap) cap = g_debug_qcap;
+    const size_t sig = (size_t)(N > 0 ? N : 1) * (size_t)((K + 255) / 256);
+    if (cap < sig) cap = sig;                       // the fit's selection words reuse the list
+    w.qcap = cap;
+    w.qlist = static_cast<uint32_t*>(take(sizeof(uint32_t) * cap));
     w.bytes = off;
     return w;
 }
@@ -113,6 +138,12 @@ size_t aaac_workspace_bytes(int mode, int64_t N, int64_t K, int64_t T) {
     return carve(nullptr, mode, N, K).bytes;
 }
 
+size_t aaac_workspace_bytes_full(int mode, int64_t N, int64_t K, int64_t T) {
+    (void)T;
+    if (mode != AAAC_INT4 && mode != AAAC_NVFP4) return 0;
+    return carve(nullptr, mode, N, K, 0, true).bytes;
+}
+
 int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
                    uint32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
     if (!X || !I) return AAAC_ERR_NULL;
@@ -121,7 +152,7 @@ int aaac_act_stats(const void* X, int64_t T, int64_t K, int64_t ldx, float* I, i
     // only the small regions are used; size the check for a 1-row layer of this width
     int rc = check_ws(ws, ws_bytes, carve(nullptr, AAAC_NVFP4, 1, K).bytes);
     if (rc) return rc;
-    Workspace w = carve(ws, AAAC_NVFP4, 1, K);
+    Workspace w = carve(ws, AAAC_NVFP4, 1, K, ws_bytes);
     return launch_act_stats(static_cast<const uint16_t*>(X), T, K, ldx, I, accumulate, dev_status, w,
                             static_cast<cudaStream_t>(stream)) == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
 }
@@ -165,7 +196,7 @@ int prepare_fit_layer(const aaac_layer& L, int mode, int init, uint32_t* dev_sta
         I = w.I;
     }
     if (launch_scales(Wp, L.N, L.K, L.ldw, mode, L.scales, L.tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
-    if (launch_init(Wp, L.N, L.K, L.ldw, mode, init, L.scales, L.T01, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (launch_init(Wp, L.N, L.K, L.ldw, mode, init, L.scales, L.T01, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
     *I_used = I;
     return AAAC_OK;
 }
@@ -184,7 +215,7 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
     int rc = AAAC_OK;
     for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
         const aaac_layer& L = layers[l];
-        const Workspace w = carve(L.ws, mode, L.N, L.K);
+        const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
         const float* I = nullptr;
         rc = prepare_fit_layer(L, mode, init, dev_status, w, st, &I);
         args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, w};
@@ -241,7 +272,7 @@ int aaac_pack_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, in
     if (!aligned(I, 16) || !aligned(codes, 16) || !aligned(T01_bf16, 2)) return AAAC_ERR_ALIGN;
     rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
     if (rc) return rc;
-    Workspace w = carve(ws, mode, N, K);
+    Workspace w = carve(ws, mode, N, K, ws_bytes);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the pack pass uses only the block counter and its own result fields of the control block
     if (cudaMemsetAsync(&w.ctrl->done, 0, sizeof(uint32_t), st) != cudaSuccess) return AAAC_ERR_CUDA;
@@ -329,6 +360,7 @@ int aaac_quantize_layer_host(const void* W_host, int64_t N, int64_t K, int mode,
     if (rc) return rc;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return AAAC_ERR_CUDA;
     if (hstatus & AAAC_DEV_TIMEOUT) return AAAC_ERR_TIMEOUT;
+    if (hstatus & AAAC_DEV_SCRATCH) return AAAC_ERR_WORKSPACE;
     return (hstatus & AAAC_DEV_NONFINITE) ? AAAC_ERR_NONFINITE : AAAC_OK;
 }
 
@@ -380,6 +412,11 @@ int aaac_quantize_layer_host_async(const void* W_host, int64_t N, int64_t K, int
     back(err_out_host, h.err, 16);
     back(status_host, h.status, 4);
     return e == cudaSuccess ? AAAC_OK : AAAC_ERR_CUDA;
+}
+
+int aaac_debug_quantile_cap(size_t entries) {
+    g_debug_qcap = entries;
+    return AAAC_OK;
 }
 
 int aaac_debug_fit_wait(int extra_arrivals, unsigned spin_limit) {

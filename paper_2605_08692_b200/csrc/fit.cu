@@ -806,7 +806,7 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
         return launch_variant<AAAC_NVFP4, 16, NW, REP, KIND>(p, (unsigned)grid, st);
     };
     // the three rotating sum buffers start at zero
-    static_assert(sizeof(unsigned long long) * 3 * kAccBuffer <= sizeof(double) * 2 * kMaxBlocks * kPartStride, "the sum buffers live in the block-partial region");
+    static_assert(sizeof(unsigned long long) * 3 * kAccBuffer <= sizeof(double) * kMaxBlocks * kPartStride, "the sum buffers live in the block-partial region");
     cudaError_t em = cudaMemsetAsync(p.acc, 0, sizeof(unsigned long long) * 3 * kAccBuffer, st);
     if (em != cudaSuccess) return em;
     if (n_inner == 1) return launch(std::integral_constant<int, kRounds>{});

@@ -24,10 +24,12 @@ namespace aaac {
 
 namespace {
 
-__device__ __forceinline__ uint32_t float_key(float f) {      // order-preserving
-    const uint32_t u = __float_as_uint(f);
+__device__ __forceinline__ uint32_t float_key(float f) {      // order-preserving; -0 and +0 share a key
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
+constexpr uint32_t kSlotOver = 0x40u;      // bin -> slot table: the slot's candidates have no room in the list
 __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
@@ -112,11 +114,13 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     __shared__ uint32_t cnt[kQReq];
     __shared__ unsigned long long base[kQReq];
     __shared__ uint32_t nbuf;
+    __shared__ uint32_t okmin[kQReq], okmax[kQReq];       // smallest / largest key of the slots without list space
     const int tid = threadIdx.x, lane = tid & 31;
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(slot_of_bin);
         for (int i = tid; i < kQBins / 4; i += blockDim.x) sm[i] = src[i];
         if (tid == 0) nbuf = 0;
+        if (tid < kQReq) { okmin[tid] = 0xFFFFFFFFu; okmax[tid] = 0u; }
     }
     __syncthreads();
     const uint8_t* sm_slot = reinterpret_cast<const uint8_t*>(sm);
@@ -171,9 +175,18 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
                 const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
                 const uint32_t s = sm_slot[qbin(x)];
                 if (s != 0xFFu) {
-                    const uint32_t pos = atomicAdd(&nbuf, 1u);
-                    buf_key[pos] = float_key(x);
-                    buf_slot[pos] = (uint8_t)s;
+                    if (s & kSlotOver) {
+                        // no list space for this slot: keep only the extremes of its keys (lanes with the
+                        // same slot combine first, so that a heavy bin costs one atomic per warp step)
+                        const uint32_t key = float_key(x), sl = s & (kSlotOver - 1u);
+                        const unsigned peers = __match_any_sync(__activemask(), sl);
+                        const uint32_t mn = __reduce_min_sync(peers, key), mx = __reduce_max_sync(peers, key);
+                        if (lane == __ffs(peers) - 1) { atomicMin(&okmin[sl], mn); atomicMax(&okmax[sl], mx); }
+                    } else {
+                        const uint32_t pos = atomicAdd(&nbuf, 1u);
+                        buf_key[pos] = float_key(x);
+                        buf_slot[pos] = (uint8_t)s;
+                    }
                 }
             }
         }
@@ -184,13 +197,18 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
         ok = okn;
     }
     flush();
+    if (tid < kQReq && okmin[tid] <= okmax[tid]) {
+        atomicMin(&ctrl->slot_kmin[tid], okmin[tid]);
+        atomicMax(&ctrl->slot_kmax[tid], okmax[tid]);
+    }
 }
 
 // one block of 1024 threads: prefix sum, bin + local rank of every request, slots.  Every thread
 // keeps its chunk of 16 bins in registers; the thread whose chunk holds a requested rank walks
 // those registers (no dependent memory reads), and the bin -> slot table is cleared by word stores.
 __global__ void __launch_bounds__(1024)
-quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __restrict__ slot_of_bin) {
+quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __restrict__ slot_of_bin,
+                     unsigned long long qcap) {
     __shared__ unsigned long long chunk[1024];
     __shared__ unsigned long long req_rank[kQReq];
     __shared__ int req_bin[kQReq];
@@ -272,27 +290,31 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __r
         req_first[tid] = first;
     }
     __syncthreads();
-    if (tid < kQReq) {
-        uint32_t slot = 0;
+    __shared__ uint32_t slot_of_req[kQReq];
+    if (tid == 0) {
+        // slots in order of first appearance; a slot gets list space while the list has room for all
+        // of its bin's weights, otherwise it is marked and only the extremes of its keys will be kept
+        uint32_t ns = 0;
         unsigned long long off = 0;
-        const int first = req_first[tid];
-        for (int q = 0; q < first; ++q)
-            if (req_first[q] == q) { ++slot; off += req_cnt[q]; }
-        ctrl->req_slot[tid] = slot;
-        if (first == tid) {
-            slot_of_bin[req_bin[tid]] = (uint8_t)slot;
-            ctrl->slot_off[slot] = off;
-            ctrl->slot_fill[slot] = 0;
+        for (int q = 0; q < kQReq; ++q) {
+            if (req_first[q] != q) { slot_of_req[q] = slot_of_req[req_first[q]]; continue; }
+            const bool fits = off + req_cnt[q] <= qcap;
+            slot_of_req[q] = ns;
+            ctrl->slot_off[ns] = off;
+            ctrl->slot_fill[ns] = 0;
+            ctrl->slot_over[ns] = fits ? 0u : 1u;
+            ctrl->slot_kmin[ns] = 0xFFFFFFFFu;
+            ctrl->slot_kmax[ns] = 0u;
+            slot_of_bin[req_bin[q]] = (uint8_t)(fits ? ns : (ns | kSlotOver));
+            if (fits) off += req_cnt[q];
+            ++ns;
         }
-        if (tid == kQReq - 1) {
-            uint32_t ns = 0;
-            unsigned long long tot = 0;
-            for (int q = 0; q < kQReq; ++q)
-                if (req_first[q] == q) { ++ns; tot += req_cnt[q]; }
-            ctrl->slot_off[ns] = tot;
-            ctrl->nslots = ns;
-        }
+        ctrl->slot_off[ns] = off;
+        ctrl->nslots = ns;
+        ctrl->scratch_short = 0u;
     }
+    __syncthreads();
+    if (tid < kQReq) ctrl->req_slot[tid] = slot_of_req[tid];
 }
 
 // one block per slot: radix select of every request that lives in this slot.
@@ -315,6 +337,16 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     __shared__ uint32_t sh_or, sh_and, sh_cnt, sh_min;
     const uint32_t slot = blockIdx.x;
     if (slot >= ctrl->nslots) return;
+    if (ctrl->slot_over[slot]) {
+        // the bin's weights had no room in the list: if they all share one value, that value is every
+        // order statistic of the bin; otherwise the scratch was too small for this layer
+        const uint32_t kmin = ctrl->slot_kmin[slot], kmax = ctrl->slot_kmax[slot];
+        if (threadIdx.x < kQReq && ctrl->req_slot[threadIdx.x] == slot) {
+            if (kmin == kmax) ctrl->rank_val[threadIdx.x] = key_float(kmin);
+            else { ctrl->rank_val[threadIdx.x] = 0.f; ctrl->scratch_short = 1u; }
+        }
+        return;
+    }
     if (threadIdx.x < kQReq) {
         req_slot[threadIdx.x] = ctrl->req_slot[threadIdx.x];
         req_local[threadIdx.x] = ctrl->req_local[threadIdx.x];
@@ -458,8 +490,9 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
 }
 
 // entry e uses requests 2e (lower neighbour) and 2e+1 (upper neighbour)
-__global__ void quantile_finish_kernel(Ctrl* ctrl) {
+__global__ void quantile_finish_kernel(Ctrl* ctrl, uint32_t* dev_status) {
     const int e = threadIdx.x;
+    if (e == 0 && ctrl->scratch_short && dev_status) atomicOr(dev_status, AAAC_DEV_SCRATCH);
     if (e >= 2 * kM) return;
     const double lo = (double)ctrl->rank_val[2 * e], hi = (double)ctrl->rank_val[2 * e + 1];
     const double v = __dadd_rn(lo, __dmul_rn(ctrl->frac[e], __dsub_rn(hi, lo)));
@@ -493,7 +526,7 @@ __global__ void grid_init_kernel(Ctrl* ctrl, int mode, const float* T01_user) {
 }  // namespace
 
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
-                        const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st) {
+                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
     if (init != AAAC_INIT_QUANTILE) {
         grid_init_kernel<<<1, 32, 0, st>>>(ws.ctrl, mode, init == AAAC_INIT_USER ? T01_user : nullptr);
         note_launch();
@@ -530,7 +563,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
         quantile_hist_kernel<AAAC_NVFP4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
         note_launch();
     }
-    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qslot_of_bin);
+    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qslot_of_bin, (unsigned long long)ws.qcap);
     note_launch();
     const int blocks1 = sm_count() * 4;
     if (mode == AAAC_INT4)
@@ -540,7 +573,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     note_launch();
     quantile_select_kernel<<<kQReq, 1024, 0, st>>>(ws.ctrl, ws.qlist);
     note_launch();
-    quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl);
+    quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl, dev_status);
     note_launch();
     return cudaGetLastError();
 }

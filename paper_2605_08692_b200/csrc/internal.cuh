@@ -45,6 +45,9 @@ struct Ctrl {
     uint32_t nslots;
     unsigned long long slot_off[kQReq + 1];
     uint32_t slot_fill[kQReq];
+    uint32_t slot_over[kQReq];      // the slot's candidates did not fit the list: only their smallest and largest key are kept
+    uint32_t slot_kmin[kQReq], slot_kmax[kQReq];
+    uint32_t scratch_short;         // an order statistic could not be found within the scratch given
     // pack results
     double pack_err[2];
     unsigned long long pack_stats[4];
@@ -52,14 +55,14 @@ struct Ctrl {
 
 struct Workspace {
     Ctrl* ctrl;
-    double* part;            // [2][kMaxBlocks][kPartStride]
-    float* rinv;             // [N*K/g]  INT4 reciprocal scales
+    double* part;            // [kMaxBlocks][kPartStride]: the pack pass's block partials; the fit rounds' sum buffers
+    float* rinv;             // [N*K/g]  INT4 reciprocal scales (one element in NVFP4 mode)
     float* I;                // [K] importance computed from X
     double* act_part;        // [kActMaxSplits][K]
     uint32_t* qhist;         // [kQBins]
-    unsigned long long* qprefix;   // [kQBins + 1]
     uint8_t* qslot_of_bin;   // [kQBins]
-    uint32_t* qlist;         // [N*K]  candidates of the quantile selection; afterwards the fit's selection bits [N][ceil(K/256)]
+    uint32_t* qlist;         // [qcap] candidates of the quantile selection; afterwards the fit's selection bits [N][ceil(K/256)]
+    size_t qcap;             // entries of qlist
     size_t bytes;
 };
 
@@ -112,7 +115,8 @@ cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ld
 cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, void* scales,
                           float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
-                        const void* scales, const float* T01_user, const Workspace& ws, cudaStream_t st);
+                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+int act_splits_max(int64_t K);    // most row strips launch_act_stats uses for K input channels (sizes its partials)
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
                               const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st);

@@ -142,6 +142,46 @@ def test_quantile_start_tables_on_degenerate_value_sets(mode, kind):
     assert table_close(host(r2["T01"]), o["T"])[0]
 
 
+def test_quantile_start_when_a_bin_does_not_fit_the_candidate_list():
+    """The candidate list of the quantile start is bounded.  A bin whose weights do not fit is
+    still answered exactly when they all share one value (constant and sparse layers); when they
+    do not, AAAC_DEV_SCRATCH is set (and the host-buffer call returns AAAC_ERR_WORKSPACE), and a
+    workspace of the full size never falls short."""
+    # (a) the default capacity on a layer whose weights take three values (each bin far over capacity)
+    rng = np.random.default_rng(5)
+    N, K = 512, 4096
+    vals = rng.choice(np.array([-1.0, 0.0, 1.0], np.float32), size=(N, K), p=[0.3, 0.4, 0.3])
+    vals[:, ::16] = 1.0                                     # every group's largest magnitude: one scale for all
+    W = synth.f32_to_bf16_bits(vals)
+    I = np.ones(K, np.float32)
+    for mode in (INT4, NVFP4):
+        g = 128 if mode == INT4 else 16
+        s, ts = oracle.scales(W, mode, g)
+        want = oracle.init_quantile(oracle.normalise(W, mode, g, s, ts)).astype(np.float32)
+        assert binding.workspace_bytes(mode, N, K) < W.nbytes * 4      # bounded: the full list alone would be 4 N K bytes
+        r = run_fit(W, mode, I, 0, binding.INIT_QUANTILE)
+        assert int(r["status"].item()) == 0
+        assert np.array_equal(host(r["T01"]), want), (host(r["T01"]), want)
+    # (b) a forced small capacity on an ordinary layer: several values per bin cannot be resolved
+    W2, X2 = layer(NVFP4, 300, 768, name="qcap")
+    I2 = oracle.act_stats(X2)
+    ref = run_fit(W2, NVFP4, I2, 2, binding.INIT_QUANTILE)
+    try:
+        binding.debug_quantile_cap(1000)
+        bad = run_fit(W2, NVFP4, I2, 2, binding.INIT_QUANTILE)
+        torch.cuda.synchronize()
+        assert int(bad["status"].item()) & binding.DEV_SCRATCH
+    finally:
+        binding.debug_quantile_cap(0)
+    # (c) the full-size workspace and the default one give the same start tables and fit
+    Wd = dev_bf16(W2)
+    Id = torch.from_numpy(I2).to(DEV)
+    full = binding.quantize_layer(Wd, NVFP4, I=Id, n_outer=2, init=binding.INIT_QUANTILE,
+                                  ws=binding.alloc_workspace(NVFP4, 300, 768, full=True))
+    assert int(full["status"].item()) == 0
+    assert torch.equal(full["T01"], ref["T01"]) and torch.equal(full["codes"], ref["codes"])
+
+
 def test_user_tables_and_nonfinite_weights():
     W, X = layer(INT4, 16, 256, name="user")
     I = oracle.act_stats(X)
