@@ -17,11 +17,12 @@
 // the number of groups with E0 == E1 exactly (among those re-evaluated), of weights exactly
 // half-way between two different entries of their table, and of groups re-evaluated in double.
 //
-// Thread mapping and pipeline as in the fit rounds: a block of NW warps takes items of 4 NW rows x
-// 256 columns in contiguous ranges, a warp 4 rows, a lane 8 adjacent columns (one 128-bit load per
-// row, one 32-bit store of 8 codes); a row's registers are refilled from the next item as soon as
-// it is unpacked, the lookups of row u + 1 are issued ahead of the arithmetic of row u, and the two
-// errors travel as one packed FP32 pair.
+// Thread mapping.  The pass keeps no bins, so its lookup tables (512 bins) leave room for two
+// blocks of 12 warps per SM, and memory and table latency are hidden by the number of warps rather
+// than by a hand-built pipeline: a warp walks down the rows of one 256-column slab (so its eight
+// importances stay in registers), one row at a time, the next row's load in flight; a lane takes 8
+// adjacent columns (one 128-bit load per row, one 32-bit store of 8 codes); the two errors travel
+// as one packed FP32 pair.
 // Error sums go through one partial per block, added in block order by the last block to finish.
 #include "lookup.cuh"
 
@@ -30,7 +31,10 @@ namespace aaac {
 namespace {
 
 // warps per block (both instances run without register spills at 12; 16 is no faster)
-constexpr int pack_warps(int) { return 12; }
+#ifndef AAAC_PACK_WARPS
+#define AAAC_PACK_WARPS 8
+#endif
+constexpr int pack_warps(int) { return AAAC_PACK_WARPS; }
 constexpr int kPackRep = 16;          // one copy of the {J_low, thr} table per lane of a half-warp: no conflicts
 
 struct PackParams {
@@ -45,7 +49,6 @@ struct PackParams {
     uint16_t* T01_bf16;
     uint8_t* codes;
     uint8_t* sigma_bits;          // [N][K / 128] when the selection group is 16 inside a scale group of 128; else null
-    int items, per_block, nrb;
 };
 
 // The rare path of a row, out of line so that the hot loop holds a single call: for the lanes that
@@ -102,14 +105,16 @@ __device__ __noinline__ Rare8 rare_groups(const FitTables* S, Row8 r, int flags)
     return out;
 }
 
+constexpr int kPackBins = 512;        // uniform bins of the per-bin table on (-8, 8): width 1/32
+constexpr int kPackBlocksPerSM = 2;
+
 template <int MODE, int SEL, int NW, int REP>
-__global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
+__global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const PackParams p) {
+    constexpr int NB = kPackBins;
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;      // scale group
     constexpr int LPG = SEL / 8;                         // lanes per selection group
     static_assert(SEL == G || SEL == 16, "separate selection bits are laid out for groups of 16");
-    constexpr int R = kRowsPerWarp;
-    constexpr int kRowsPerItem = R * NW;
-    constexpr int kLut1Bytes = REP * kNBins * 8;
+    constexpr int kLut1Bytes = REP * NB * 8;
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ FitTables S;
     __shared__ float slut[128];                      // NVFP4: s_eff per E4M3 code
@@ -140,13 +145,14 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
     }
     __syncthreads();
     if (blockIdx.x == 0 && tid < 2 * kM) p.T01_bf16[tid] = (uint16_t)(__float_as_uint((float)S.Td[tid]) >> 16);
-    build_tables<MODE, NW, REP>(S, dyn);
+    build_tables<MODE, NW, REP, NB>(S, dyn);
 
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
     const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;
     const uint32_t lut2_addr = sm_base + kLut1Bytes;                // the {P, Q} table
-    constexpr float kMagic = 512.f + 1.5f * (float)(1 << 23) / (float)(REP * 8);
-    constexpr uint32_t kBinMask = (uint32_t)(kNBins - 1) * (REP * 8);
+    constexpr float kBinsPerUnit = (float)(NB / 16);
+    constexpr float kMagic = (float)(NB / 2) + 1.5f * (float)(1 << 23) / (float)(REP * 8);
+    constexpr uint32_t kBinMask = (uint32_t)(NB - 1) * (REP * 8);
     // near-tie bound (see fit.cu): |E0 - E1| <= g1 (E0 + E1) + g2 sum I sends the group to the double path
     const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
 
@@ -155,49 +161,21 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
 
     const int N = (int)p.N, K = (int)p.K;
     const int Gr = K / G;
-    const int it0 = blockIdx.x * p.per_block;
-    const int it1 = min(p.items, it0 + p.per_block);
+    const int slabs = (K + 255) >> 8;
+    // Warp w of the grid takes slab w mod slabs and, of the warps that share that slab, every
+    // (warps per slab)-th row; with fewer warps than slabs a warp takes several slabs in turn.
+    const int gw = blockIdx.x * NW + warp, nw_total = gridDim.x * NW;
 
-    // Row registers of the item being processed, refilled from the next item as soon as a row has
-    // been unpacked (as in the fit rounds).
-    uint4 v[R];
-    uint32_t sc[R];           // scale bits (sign clear): E4M3 byte or BF16 pattern
-    auto load_row = [&](int u, int slab, int rb) {
+    for (int slab = gw % slabs; slab < slabs; slab += nw_total) {
+        // the rows of the slab are dealt to the warps that share it (those with the same index mod
+        // slabs): warp number `my` of `per_slab` takes rows my, my + per_slab, ...
+        const int per_slab = nw_total >= slabs ? (nw_total - (gw % slabs) + slabs - 1) / slabs : 1;
+        const int my = nw_total >= slabs ? gw / slabs : 0;
         const int col0 = slab * 256 + lane * 8;
-        const int row = rb * kRowsPerItem + warp * R + u;
-        v[u] = make_uint4(0, 0, 0, 0);
-        sc[u] = 0u;
-        if (col0 < K && row < N) {
-            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
-            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
-            if (MODE == AAAC_NVFP4) sc[u] = reinterpret_cast<const uint8_t*>(p.scales)[gi];
-            else sc[u] = reinterpret_cast<const uint16_t*>(p.scales)[gi];
-        }
-    };
-
-    int cur_slab = -1;
-    uint64_t II[8];           // {I, I} of the lane's eight columns
-    float isum = 0.f;         // g2 * sum of I over the lane's selection group (rounded up a little)
-    bool col_ok = false;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) II[j] = 0ull;
-
-    int slab = it0 / p.nrb, rb = it0 - slab * p.nrb;
-    int nslab = slab, nrb = rb;
-    if (it0 < it1) {
-#pragma unroll
-        for (int u = 0; u < R; ++u) load_row(u, slab, rb);
-    }
-    for (int item = it0; item < it1; ++item) {
-        slab = nslab;
-        rb = nrb;
-        if (++nrb == p.nrb) { nrb = 0; ++nslab; }
-        const bool more = item + 1 < it1;
-        const int col0 = slab * 256 + lane * 8;
-        if (slab != cur_slab) {
-            cur_slab = slab;
-            col_ok = col0 < K;
-            isum = 0.f;
+        const bool col_ok = col0 < K;
+        uint64_t II[8];                       // {I, I} of the lane's eight columns
+        float isum = 0.f;                     // g2 * sum of I over the lane's selection group (rounded up a little)
+        {
             float Iv[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) Iv[j] = 0.f;
@@ -213,62 +191,53 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
             for (int o = LPG / 2; o; o >>= 1) isum += __shfl_xor_sync(0xFFFFFFFFu, isum, o);
             isum = __fmul_ru(isum * 1.0001f, g2);
         }
-        const int row0 = rb * kRowsPerItem + warp * R;
-        const int nrows = min(R, N - row0);                // rows of this warp inside the layer (may be <= 0)
-
-        // Stages of a row, the table lookups of the next row issued ahead of the arithmetic of this one:
-        //   L1(u): w~ and the loads of {J_low, thr};   L2: slot and the loads of {P, Q};
-        //   M(u):  errors, sigma, codes, stores.
-        float eitem = 0.f, eoitem = 0.f;                   // the item's share of the two error sums (this lane's groups)
-        float x[2][8];                                     // w~
-        uint2 e1v[2][8];                                   // {address of the lower interval's {P, Q} entry, thr}
-        float sval[2];                                     // scale of the row's group
-        uint32_t sbits[2];
-        uint64_t pq[8];                                    // {P, Q}, packed
-        bool tcand = false;                                // some w~ equals the breakpoint of its bin
-        auto L1 = [&](int u, int b) {
-            sbits[b] = MODE == AAAC_NVFP4 ? (sc[u] & 0x7Fu) : (sc[u] & 0x7FFFu);
-            float rinv;
+        auto load = [&](int row, uint4& v, uint32_t& sc) {
+            v = make_uint4(0, 0, 0, 0);
+            sc = 0u;
+            if (col_ok && row < N) {
+                v = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
+                const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+                if (MODE == AAAC_NVFP4) sc = reinterpret_cast<const uint8_t*>(p.scales)[gi];
+                else sc = reinterpret_cast<const uint16_t*>(p.scales)[gi];
+            }
+        };
+        uint4 vn;
+        uint32_t scn;
+        load(my, vn, scn);
+        float ef = 0.f, eof = 0.f;            // the two error sums of up to 16 rows (double arithmetic is slow: one conversion per 16 rows)
+        int nrow = 0;
+        for (int row = my; row < N; row += per_slab) {
+            const uint4 v = vn;
+            const uint32_t sbits = MODE == AAAC_NVFP4 ? (scn & 0x7Fu) : (scn & 0x7FFFu);
+            load(row + per_slab, vn, scn);                 // the next row of this warp, in flight during this one
+            float sval, rinv;
             if (MODE == AAAC_NVFP4) {
-                sval[b] = slut[sbits[b]];
-                rinv = S.rlut[sbits[b]];
+                sval = slut[sbits];
+                rinv = S.rlut[sbits];
             } else {
-                sval[b] = __uint_as_float(sbits[b] << 16);
-                rinv = sbits[b] ? __frcp_rn(sval[b]) : 0.f;     // lanes past K hold no scale
+                sval = __uint_as_float(sbits << 16);
+                rinv = sbits ? __frcp_rn(sval) : 0.f;       // lanes past K hold no scale
             }
-            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                x[b][j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[b][j], 64.f, kMagic)) & kBinMask;
-                e1v[b][j] = lds_table_u2(lut1_lane + off);
-            }
-        };
-        auto L1n = [&](int u, int b) {
-            L1(u, b);
-            if (more) load_row(u, nslab, nrb);
-        };
-        auto L2 = [&](int b) {
-            tcand = false;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float thr = __uint_as_float(e1v[b][j].y);
-                tcand |= (x[b][j] == thr);
-                pq[j] = lds_table_b64(above_addr(e1v[b][j].x, x[b][j], e1v[b][j].y));
-            }
-        };
-        auto M = [&](int row, int b) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            float x[8];
+            uint64_t pq[8];
+            bool tcand = false;                             // some w~ equals the breakpoint of its bin
             uint64_t e01 = 0ull;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const uint64_t u01 = diff2(x[b][j], pq[j]);
+                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
+                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask;
+                const uint2 e = lds_table_u2(lut1_lane + off);
+                tcand |= (x[j] == __uint_as_float(e.y));
+                pq[j] = lds_table_b64(above_addr(e.x, x[j], e.y));
+                const uint64_t u01 = diff2(x[j], pq[j]);
                 e01 = fma2(mul2(II[j], u01), u01, e01);
             }
             float e0 = lo2(e01), e1 = hi2(e01);
 #pragma unroll
-            for (int s = LPG / 2; s; s >>= 1) {
-                e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, s);
-                e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, s);
+            for (int s2 = LPG / 2; s2; s2 >>= 1) {
+                e0 += __shfl_xor_sync(0xFFFFFFFFu, e0, s2);
+                e1 += __shfl_xor_sync(0xFFFFFFFFu, e1, s2);
             }
             const float es = e0 + e1;
             const float tau = __fmaf_ru(es, g1, isum);
@@ -279,7 +248,7 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
                 // near-ties, poisoned slots and weights that sit on a breakpoint (rare, out of line)
                 Row8 r;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { r.x[j] = x[b][j]; r.I[j] = lo2(II[j]); r.hint[j] = interval_hint(S, pq[j]); }
+                for (int j = 0; j < 8; ++j) { r.x[j] = x[j]; r.I[j] = lo2(II[j]); r.hint[j] = interval_hint(S, pq[j]); }
                 const Rare8 ex = rare_groups<LPG>(&S, r, (near ? kNear : 0) | (tcand ? kTieCand : 0) | (sg ? kFastSigma : 0));
                 if (near) {
 #pragma unroll
@@ -301,12 +270,13 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
                 if (col_ok && (lane & 15) == 0)
                     p.sigma_bits[(size_t)row * (size_t)(K >> 7) + (uint32_t)col0 / 128u] = (uint8_t)(bb >> (lane >> 1));
             }
-            if (!col_ok) return;
+            if (!col_ok) continue;
             if ((lane % LPG) == 0) {
                 // both error sums from the group's smaller error: sum I (w - w^)^2 = s^2 sum I (w~ - T)^2
-                eitem += emin;
-                eoitem = __fmaf_rn(emin, __fmul_rn(sval[b], sval[b]), eoitem);
+                ef += emin;
+                eof = __fmaf_rn(emin, __fmul_rn(sval, sval), eof);
             }
+            if (++nrow == 16) { Eacc += (double)ef; Eout += (double)eof; ef = 0.f; eof = 0.f; nrow = 0; }
             // codes (Eq. 6): the entry index rides in the low mantissa bits of the chosen constant
             uint32_t word = 0;
 #pragma unroll
@@ -319,41 +289,13 @@ __global__ void __launch_bounds__(NW * 32, 1) pack_kernel(const PackParams p) {
             if (SEL == G && (lane % LPG) == 0) {
                 const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
                 if (MODE == AAAC_NVFP4)
-                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits[b] | (sg ? 0x80u : 0u));
+                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
                 else
-                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits[b] | (sg ? 0x8000u : 0u));
-            }
-        };
-
-        if (nrows == R) {
-            L1n(0, 0);
-#pragma unroll
-            for (int u = 0; u < R; ++u) {
-                if (u + 1 < R) L1n(u + 1, (u + 1) & 1);
-                L2(u & 1);
-                M(row0 + u, u & 1);
-            }
-        } else {
-            // ragged last row block of the layer: row by row, then refill all rows
-            uint4 vr[R];
-            uint32_t sr[R];
-#pragma unroll
-            for (int t = 0; t < R; ++t) { vr[t] = v[t]; sr[t] = sc[t]; }
-            for (int u = 0; u < nrows; ++u) {
-#pragma unroll
-                for (int t = 0; t < R; ++t)
-                    if (u == t) { v[0] = vr[t]; sc[0] = sr[t]; }
-                L1(0, 0);
-                L2(0);
-                M(row0 + u, 0);
-            }
-            if (more) {
-#pragma unroll
-                for (int t = 0; t < R; ++t) load_row(t, nslab, nrb);
+                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits | (sg ? 0x8000u : 0u));
             }
         }
-        Eacc += (double)eitem;
-        Eout += (double)eoitem;
+        Eacc += (double)ef;
+        Eout += (double)eof;
     }
 
     // ---- block partial of the two error sums; integer statistics by atomics ----
@@ -403,7 +345,7 @@ __global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long lo
 
 template <int MODE, int SEL>
 cudaError_t launch_pack_variant(const PackParams& p, unsigned grid, cudaStream_t st) {
-    constexpr size_t smem = (size_t)kPackRep * kNBins * 8 + kLut2Bytes;
+    constexpr size_t smem = (size_t)kPackRep * kPackBins * 8 + kLut2Bytes;
     constexpr int kPackWarps = pack_warps(MODE);
     auto kern = pack_kernel<MODE, SEL, kPackWarps, kPackRep>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -424,16 +366,14 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     p.scales = scales; p.I = I; p.tensor_scale = tensor_scale;
     p.ctrl = ws.ctrl; p.part = ws.part; p.T01_f32 = T01_f32; p.T01_bf16 = T01_bf16; p.codes = codes;
     p.sigma_bits = sigma_bits;
+    if (N > 0x7FFFFFFF || K > 0x7FFFFFFF) return cudaErrorInvalidValue;
+    // two blocks per SM; no more warps than there are (row, slab) pieces of work
     const int64_t slabs = (K + 255) / 256;
-    const int kRowsPerItem = kRowsPerWarp * pack_warps(mode);
-    const int64_t nrb = (N + kRowsPerItem - 1) / kRowsPerItem, items = slabs * nrb;
-    if (N > 0x7FFFFFFF || K > 0x7FFFFFFF || items > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    int64_t grid = sm_count();
-    if (grid > items) grid = items;
+    int64_t grid = (int64_t)sm_count() * kPackBlocksPerSM;
+    const int64_t pieces = (N * slabs + pack_warps(mode) - 1) / pack_warps(mode);
+    if (grid > pieces) grid = pieces;
     if (grid > kMaxBlocks) grid = kMaxBlocks;
-    const int64_t per_block = (items + grid - 1) / grid;
-    grid = (items + per_block - 1) / per_block;
-    p.nrb = (int)nrb; p.items = (int)items; p.per_block = (int)per_block;
+    if (grid < 1) grid = 1;
     cudaError_t e;
     if (mode == AAAC_INT4 && sel_group == 16) e = launch_pack_variant<AAAC_INT4, 16>(p, (unsigned)grid, st);
     else if (mode == AAAC_INT4) e = launch_pack_variant<AAAC_INT4, 128>(p, (unsigned)grid, st);
