@@ -54,7 +54,7 @@ def peaks():
     return 6650.0, "fallback"
 
 
-TRAFFIC_FILE = os.path.join("profiles", "fit_rounds_cfg2_gate_proj.md")
+TRAFFIC_FILE = os.path.join("profiles", "fit_batch_cfg2_full_step.md")
 
 
 def measured_traffic_per_weight():
@@ -472,8 +472,8 @@ def main():
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
                 "traffic": None if tpw is None else tpw * float(np.mean(per_launch_w)),
                 "traffic_source": None if tpw is None else f"{TRAFFIC_FILE} (a constant per weight and round from one "
-                                                           "earlier ncu capture on gate_proj, scaled to the mean launch; "
-                                                           "not measured in this run)",
+                                                           "earlier ncu capture of this workload's launch; not measured "
+                                                           "in this run)",
                 "algorithmic_bytes_per_launch": float(np.mean(per_launch_w)) * BYTES_PER_WEIGHT,
                 "avg_launch_ms": fit_ms / max(len(round_ms), 1),
                 "fit_share_of_step": fit_ms / ms_total if ms_total > 0 else None,
