@@ -218,7 +218,7 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
         const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
         const float* I = nullptr;
         rc = prepare_fit_layer(L, mode, init, dev_status, w, st, &I);
-        args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, w};
+        args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, L.T01, w};
     }
     if (rc == AAAC_OK) {
         // all rounds run in one launch per batch; the optional timing brackets the launches of this call
@@ -235,7 +235,8 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
         if (launch_fit_rounds_batch(args, n_layers, mode, sel_group, n_outer, n_inner, dev_status, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
         if (e1) cudaEventRecord(e1, st);
     }
-    for (int l = 0; l < n_layers && rc == AAAC_OK; ++l)
+    // with rounds to run the last fit launch writes the tables out itself; with none, a small kernel does
+    for (int l = 0; l < n_layers && rc == AAAC_OK && n_outer == 0; ++l)
         if (launch_export_tables(layers[l].T01, args[l].ws, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
     delete[] args;
     return rc;

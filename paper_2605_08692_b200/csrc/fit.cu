@@ -84,6 +84,7 @@ struct FitParams {
     Ctrl* ctrl;
     unsigned long long* acc;      // [3][kUsed][3] words, 128 bytes apart: fixed-point sums over the blocks, one buffer per pass in rotation
     double* err_trace;            // [n_rounds] or null
+    float* T01_out;               // [2][16] or null: the tables after the launch's last pass, as FP32
     uint32_t* dev_status;         // or null
     uint32_t* sigw;               // [N][slabs]: selection bits of a row's 256-column slab, bit = lane (n_inner > 1)
     int n_rounds;                 // passes over W in this launch
@@ -693,7 +694,10 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
         p.err_trace[p.trace_base + round] = S.tot[2 * kCells];
     __syncthreads();
   }
-    if (bid == 0 && tid < 2 * kM) p.ctrl->T[tid] = S.Td[tid];
+    if (bid == 0 && tid < 2 * kM) {
+        p.ctrl->T[tid] = S.Td[tid];
+        if (p.T01_out) p.T01_out[tid] = (float)S.Td[tid];
+    }
 }
 
 template <int MODE, int SEL, int NW, int REP, int KIND>
@@ -779,7 +783,7 @@ static bool fill_params(FitParams& p, const FitLayerArgs& a, int n_outer, uint32
     p = FitParams{};
     p.W = a.W; p.N = a.N; p.K = a.K; p.ldw = a.ldw;
     p.scales = static_cast<const uint8_t*>(a.scales); p.rinv = a.ws.rinv; p.I = a.I;
-    p.ctrl = a.ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(a.ws.part); p.err_trace = a.err_trace; p.dev_status = dev_status;
+    p.ctrl = a.ws.ctrl; p.acc = reinterpret_cast<unsigned long long*>(a.ws.part); p.err_trace = a.err_trace; p.T01_out = a.T01_out; p.dev_status = dev_status;
     p.n_rounds = n_outer; p.trace_base = 0; p.bar_base = 0u;
     p.spin_limit = g_spin_limit;
     p.sigw = a.ws.qlist;            // the quantile selection's list is free once the start tables exist
@@ -790,11 +794,11 @@ static bool fill_params(FitParams& p, const FitLayerArgs& a, int n_outer, uint32
 }
 
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
-                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
+                              const float* I, int n_outer, int n_inner, double* err_trace, float* T01_out, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st) {
     if (n_outer <= 0) return cudaSuccess;
     if (n_inner < 1 || (int64_t)n_outer * n_inner > 0x7FFFFFFF) return cudaErrorInvalidValue;
-    FitLayerArgs a{W, N, K, ldw, scales, I, err_trace, ws};
+    FitLayerArgs a{W, N, K, ldw, scales, I, err_trace, T01_out, ws};
     FitParams p;
     if (!fill_params(p, a, n_outer, dev_status)) return cudaErrorInvalidValue;
     const int64_t grid = plan_layer(p, N, K, sm_count());
@@ -847,7 +851,7 @@ cudaError_t launch_fit_rounds_batch(const FitLayerArgs* layers, int n, int mode,
             // single layers and inner refinement go through the one-layer launches
             const FitLayerArgs& a = layers[at];
             cudaError_t e = launch_fit_rounds(a.W, a.N, a.K, a.ldw, mode, sel_group, a.scales, a.I, n_outer, n_inner,
-                                              a.err_trace, dev_status, a.ws, st);
+                                              a.err_trace, a.T01_out, dev_status, a.ws, st);
             if (e != cudaSuccess) return e;
             at += 1;
             continue;

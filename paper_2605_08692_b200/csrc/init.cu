@@ -203,12 +203,17 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     }
 }
 
+struct Requests {                     // the order statistics asked for (host-computed from N K alone)
+    unsigned long long rank[kQReq];
+    double frac[2 * kM];
+};
+
 // one block of 1024 threads: prefix sum, bin + local rank of every request, slots.  Every thread
 // keeps its chunk of 16 bins in registers; the thread whose chunk holds a requested rank walks
 // those registers (no dependent memory reads), and the bin -> slot table is cleared by word stores.
 __global__ void __launch_bounds__(1024)
 quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __restrict__ slot_of_bin,
-                     unsigned long long qcap) {
+                     unsigned long long qcap, const Requests rq) {
     __shared__ unsigned long long chunk[1024];
     __shared__ unsigned long long req_rank[kQReq];
     __shared__ int req_bin[kQReq];
@@ -230,7 +235,9 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __r
     unsigned long long s = 0;
 #pragma unroll
     for (int i = 0; i < per; ++i) s += h[i];
-    if (tid < kQReq) req_rank[tid] = ctrl->rank[tid];
+    if (tid < kQReq) req_rank[tid] = rq.rank[tid];
+    if (tid < 2 * kM) ctrl->frac[tid] = rq.frac[tid];
+    if (tid == 0) ctrl->done = 0u;                          // blocks of the selection kernel that have finished
     {
         uint32_t* clr = reinterpret_cast<uint32_t*>(slot_of_bin);
 #pragma unroll
@@ -290,10 +297,39 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __r
         req_first[tid] = first;
     }
     __syncthreads();
+    // slots in order of first appearance among the requests.  A slot gets list space while the list has
+    // room for all of its bin's weights; otherwise it is marked and only the extremes of its keys will
+    // be kept.  When everything fits (the usual case) the 64 requests work out their slots side by side.
     __shared__ uint32_t slot_of_req[kQReq];
-    if (tid == 0) {
-        // slots in order of first appearance; a slot gets list space while the list has room for all
-        // of its bin's weights, otherwise it is marked and only the extremes of its keys will be kept
+    __shared__ int all_fit;
+    if (tid < kQReq) {
+        uint32_t slot = 0, ns = 0;
+        unsigned long long off = 0, tot = 0;
+        const int first = req_first[tid];
+        for (int q = 0; q < kQReq; ++q) {
+            if (req_first[q] != q) continue;
+            if (q < first) { ++slot; off += req_cnt[q]; }
+            ++ns;
+            tot += req_cnt[q];
+        }
+        if (tid == 0) all_fit = tot <= qcap;
+        if (tot <= qcap) {
+            slot_of_req[tid] = slot;
+            if (first == tid) {
+                ctrl->slot_off[slot] = off;
+                ctrl->slot_fill[slot] = 0;
+                ctrl->slot_over[slot] = 0u;
+                slot_of_bin[req_bin[tid]] = (uint8_t)slot;
+            }
+            if (tid == kQReq - 1) {
+                ctrl->slot_off[ns] = tot;
+                ctrl->nslots = ns;
+                ctrl->scratch_short = 0u;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && !all_fit) {
         uint32_t ns = 0;
         unsigned long long off = 0;
         for (int q = 0; q < kQReq; ++q) {
@@ -327,8 +363,7 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __r
 //  - The two neighbours that one table entry interpolates between are consecutive ranks: the
 //    second is the first's key again, or the smallest larger key -- one sweep instead of a
 //    second selection.
-__global__ void __launch_bounds__(1024)
-quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
+__device__ __forceinline__ void select_slot(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     __shared__ uint32_t hist[256];
     __shared__ uint32_t sh_prefix, sh_mask;
     __shared__ unsigned long long sh_k;
@@ -489,24 +524,27 @@ quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list) {
     }
 }
 
-// entry e uses requests 2e (lower neighbour) and 2e+1 (upper neighbour)
-__global__ void quantile_finish_kernel(Ctrl* ctrl, uint32_t* dev_status) {
+// One block per slot; the last block to finish interpolates the table entries: entry e uses requests
+// 2e (lower neighbour) and 2e+1 (upper neighbour), in double, rounded to FP32.
+__global__ void __launch_bounds__(1024)
+quantile_select_kernel(Ctrl* ctrl, const uint32_t* __restrict__ list, uint32_t* dev_status) {
+    __shared__ int last;
+    select_slot(ctrl, list);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(&ctrl->done, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
     const int e = threadIdx.x;
-    if (e == 0 && ctrl->scratch_short && dev_status) atomicOr(dev_status, AAAC_DEV_SCRATCH);
+    if (e == 0) {
+        ctrl->done = 0u;
+        if (__ldcg(&ctrl->scratch_short) && dev_status) atomicOr(dev_status, AAAC_DEV_SCRATCH);
+    }
     if (e >= 2 * kM) return;
-    const double lo = (double)ctrl->rank_val[2 * e], hi = (double)ctrl->rank_val[2 * e + 1];
+    const double lo = (double)__ldcg(&ctrl->rank_val[2 * e]), hi = (double)__ldcg(&ctrl->rank_val[2 * e + 1]);
     const double v = __dadd_rn(lo, __dmul_rn(ctrl->frac[e], __dsub_rn(hi, lo)));
     ctrl->T[e] = (double)(float)v;
-}
-
-struct Requests {
-    unsigned long long rank[kQReq];
-    double frac[2 * kM];
-};
-__global__ void set_requests_kernel(Ctrl* ctrl, const Requests rq) {
-    const int t = threadIdx.x;
-    if (t < kQReq) ctrl->rank[t] = rq.rank[t];
-    if (t < 2 * kM) ctrl->frac[t] = rq.frac[t];
 }
 
 __global__ void grid_init_kernel(Ctrl* ctrl, int mode, const float* T01_user) {
@@ -549,8 +587,6 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
         rq.frac[e] = pos - lo;
     }
     cudaError_t e;
-    set_requests_kernel<<<1, 64, 0, st>>>(ws.ctrl, rq);
-    note_launch();
     if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) return e;
     const int blocks = sm_count() * 3;
     const size_t sm0 = kQBins * sizeof(uint32_t);
@@ -563,7 +599,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
         quantile_hist_kernel<AAAC_NVFP4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
         note_launch();
     }
-    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qslot_of_bin, (unsigned long long)ws.qcap);
+    quantile_plan_kernel<<<1, 1024, 0, st>>>(ws.ctrl, ws.qhist, ws.qslot_of_bin, (unsigned long long)ws.qcap, rq);
     note_launch();
     const int blocks1 = sm_count() * 4;
     if (mode == AAAC_INT4)
@@ -571,9 +607,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     else
         quantile_collect_kernel<AAAC_NVFP4><<<blocks1, 256, kQBins, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qslot_of_bin, ws.qlist);
     note_launch();
-    quantile_select_kernel<<<kQReq, 1024, 0, st>>>(ws.ctrl, ws.qlist);
-    note_launch();
-    quantile_finish_kernel<<<1, 32, 0, st>>>(ws.ctrl, dev_status);
+    quantile_select_kernel<<<kQReq, 1024, 0, st>>>(ws.ctrl, ws.qlist, dev_status);
     note_launch();
     return cudaGetLastError();
 }

@@ -118,7 +118,7 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
                         const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
 int act_splits_max(int64_t K);    // most row strips launch_act_stats uses for K input channels (sizes its partials)
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
-                              const float* I, int n_outer, int n_inner, double* err_trace, uint32_t* dev_status,
+                              const float* I, int n_outer, int n_inner, double* err_trace, float* T01_out, uint32_t* dev_status,
                               const Workspace& ws, cudaStream_t st);
 // the same for several layers of one mode in a single launch (n_inner = 1; otherwise layer by layer)
 struct FitLayerArgs {
@@ -127,6 +127,7 @@ struct FitLayerArgs {
     const void* scales;
     const float* I;
     double* err_trace;
+    float* T01_out;          // where the fitted tables go as FP32 (written by the last launch), or null
     Workspace ws;
 };
 cudaError_t launch_fit_rounds_batch(const FitLayerArgs* layers, int n, int mode, int sel_group, int n_outer, int n_inner,

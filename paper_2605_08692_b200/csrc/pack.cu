@@ -49,6 +49,8 @@ struct PackParams {
     uint16_t* T01_bf16;
     uint8_t* codes;
     uint8_t* sigma_bits;          // [N][K / 128] when the selection group is 16 inside a scale group of 128; else null
+    double* err_out;              // [2] or null
+    unsigned long long* stats;    // [4] or null
 };
 
 // The rare path of a row, out of line so that the hot loop holds a single call: for the lanes that
@@ -327,20 +329,18 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
     __syncthreads();
     if (!S.is_last) return;
     __threadfence();
+    // the last block to finish adds the block partials in block order and hands the results out
     if (tid < 2) {
         double s = 0.0;
         for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(p.part + (size_t)b * kPartStride + tid);
         p.ctrl->pack_err[tid] = s;
+        if (p.err_out) p.err_out[tid] = s;
+    }
+    if (tid < 4) {
+        if (p.stats) p.stats[tid] = __ldcg(&p.ctrl->pack_stats[tid]);
+        p.ctrl->pack_stats[tid] = 0;
     }
     if (tid == 0) p.ctrl->done = 0;
-}
-
-__global__ void export_pack_kernel(Ctrl* ctrl, double* err_out, unsigned long long* stats) {
-    if (threadIdx.x < 2 && err_out) err_out[threadIdx.x] = ctrl->pack_err[threadIdx.x];
-    if (threadIdx.x < 4) {
-        if (stats) stats[threadIdx.x] = ctrl->pack_stats[threadIdx.x];
-        ctrl->pack_stats[threadIdx.x] = 0;
-    }
 }
 
 template <int MODE, int SEL>
@@ -366,6 +366,7 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     p.scales = scales; p.I = I; p.tensor_scale = tensor_scale;
     p.ctrl = ws.ctrl; p.part = ws.part; p.T01_f32 = T01_f32; p.T01_bf16 = T01_bf16; p.codes = codes;
     p.sigma_bits = sigma_bits;
+    p.err_out = err_out; p.stats = stats;
     if (N > 0x7FFFFFFF || K > 0x7FFFFFFF) return cudaErrorInvalidValue;
     // two blocks per SM; no more warps than there are (row, slab) pieces of work
     const int64_t slabs = (K + 255) / 256;
@@ -378,10 +379,7 @@ cudaError_t launch_pack(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
     if (mode == AAAC_INT4 && sel_group == 16) e = launch_pack_variant<AAAC_INT4, 16>(p, (unsigned)grid, st);
     else if (mode == AAAC_INT4) e = launch_pack_variant<AAAC_INT4, 128>(p, (unsigned)grid, st);
     else e = launch_pack_variant<AAAC_NVFP4, 16>(p, (unsigned)grid, st);
-    if (e != cudaSuccess) return e;
-    export_pack_kernel<<<1, 32, 0, st>>>(ws.ctrl, err_out, stats);
-    note_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace aaac

@@ -28,7 +28,7 @@ __device__ __forceinline__ uint32_t absmax16(uint4 v) {
 }
 
 __global__ void __launch_bounds__(256)
-absmax_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, Ctrl* ctrl) {
+absmax_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, Ctrl* ctrl, uint32_t* dev_status) {
     const int lane = threadIdx.x & 31;
     const int64_t slabs = (K + 255) / 256;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -52,14 +52,17 @@ absmax_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
     for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if (lane == 0 && m) {
         atomicMax(&ctrl->absmax_bits, m << 16);
-        if (m >= 0x7F80u) atomicOr(&ctrl->nonfinite, 1u);
+        if (m >= 0x7F80u) {
+            atomicOr(&ctrl->nonfinite, 1u);
+            if (dev_status) atomicOr(dev_status, AAAC_DEV_NONFINITE);
+        }
     }
 }
 
 template <int MODE>
 __global__ void __launch_bounds__(256)
 scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw, void* __restrict__ scales,
-              float* __restrict__ rinv, float* __restrict__ tensor_scale, Ctrl* ctrl) {
+              float* __restrict__ rinv, float* __restrict__ tensor_scale, Ctrl* ctrl, uint32_t* dev_status) {
     constexpr int G = MODE == AAAC_INT4 ? 128 : 16;
     constexpr int LPG = G / 8;                         // lanes per group
     const int lane = threadIdx.x & 31;
@@ -120,11 +123,10 @@ scales_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t ldw,
         }
       }
     }
-    if (bad) atomicOr(&ctrl->nonfinite, 1u);
-}
-
-__global__ void publish_status_kernel(const Ctrl* ctrl, uint32_t* dev_status) {
-    if (ctrl->nonfinite) atomicOr(dev_status, AAAC_DEV_NONFINITE);
+    if (bad) {
+        atomicOr(&ctrl->nonfinite, 1u);
+        if (dev_status) atomicOr(dev_status, AAAC_DEV_NONFINITE);
+    }
 }
 
 }  // namespace
@@ -133,22 +135,15 @@ cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, 
                           float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
     const int blocks = sm_count() * 8;
     if (mode == AAAC_NVFP4) {
-        absmax_kernel<<<blocks, 256, 0, st>>>(W, N, K, ldw, ws.ctrl);
+        absmax_kernel<<<blocks, 256, 0, st>>>(W, N, K, ldw, ws.ctrl, dev_status);
         note_launch();
-        scales_kernel<AAAC_NVFP4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, nullptr, tensor_scale, ws.ctrl);
+        scales_kernel<AAAC_NVFP4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, nullptr, tensor_scale, ws.ctrl, dev_status);
         note_launch();
     } else {
-        scales_kernel<AAAC_INT4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, ws.rinv, tensor_scale, ws.ctrl);
+        scales_kernel<AAAC_INT4><<<blocks, 256, 0, st>>>(W, N, K, ldw, scales, ws.rinv, tensor_scale, ws.ctrl, dev_status);
         note_launch();
     }
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (dev_status) {
-        publish_status_kernel<<<1, 1, 0, st>>>(ws.ctrl, dev_status);
-        note_launch();
-        e = cudaGetLastError();
-    }
-    return e;
+    return cudaGetLastError();
 }
 
 }  // namespace aaac
