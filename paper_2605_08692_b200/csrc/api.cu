@@ -195,8 +195,9 @@ int prepare_fit_layer(const aaac_layer& L, int mode, int init, uint32_t* dev_sta
             return AAAC_ERR_CUDA;
         I = w.I;
     }
-    if (launch_scales(Wp, L.N, L.K, L.ldw, mode, L.scales, L.tensor_scale, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
-    if (launch_init(Wp, L.N, L.K, L.ldw, mode, init, L.scales, L.T01, dev_status, w, st) != cudaSuccess) return AAAC_ERR_CUDA;
+    const bool fused = init == AAAC_INIT_QUANTILE;      // the scales pass counts the quantile start's histogram on its way
+    if (launch_scales(Wp, L.N, L.K, L.ldw, mode, L.scales, L.tensor_scale, dev_status, w, st, fused) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (launch_init(Wp, L.N, L.K, L.ldw, mode, init, L.scales, L.T01, dev_status, w, st, fused) != cudaSuccess) return AAAC_ERR_CUDA;
     *I_used = I;
     return AAAC_OK;
 }

@@ -33,13 +33,6 @@ constexpr uint32_t kSlotOver = 0x40u;      // bin -> slot table: the slot's cand
 __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
-// bin = floor(1024 x + 8192): one multiply-add rounded down onto 1.5 * 2^23 (where floats are
-// spaced by 1) leaves the integer in the low mantissa bits; the mask keeps any input inside the
-// table (|w~| < 8 by the scale rules, so for finite weights it changes nothing)
-__device__ __forceinline__ int qbin(float x) {
-    return (int)(__float_as_uint(__fmaf_rd(x, 1024.f, 8192.f + 12582912.f)) & (uint32_t)(kQBins - 1));
-}
-
 // reciprocal of the group's scale for the 8 weights a lane holds
 template <int MODE>
 __device__ __forceinline__ float group_rinv(const void* scales, int64_t gi, float s_t) {
@@ -170,21 +163,30 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
         fetch(vn, rn, okn);
         if (ok) {
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            // the slots of the lane's eight weights first (most rows hold no candidate at all: one test)
+            float x[8];
+            uint32_t sl[8], all = 0xFFu;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const float x = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
-                const uint32_t s = sm_slot[qbin(x)];
-                if (s != 0xFFu) {
+                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
+                sl[j] = sm_slot[qbin(x[j])];
+                all &= sl[j];
+            }
+            if (all != 0xFFu) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t s = sl[j];
+                    if (s == 0xFFu) continue;
                     if (s & kSlotOver) {
                         // no list space for this slot: keep only the extremes of its keys (lanes with the
                         // same slot combine first, so that a heavy bin costs one atomic per warp step)
-                        const uint32_t key = float_key(x), sl = s & (kSlotOver - 1u);
-                        const unsigned peers = __match_any_sync(__activemask(), sl);
+                        const uint32_t key = float_key(x[j]), so = s & (kSlotOver - 1u);
+                        const unsigned peers = __match_any_sync(__activemask(), so);
                         const uint32_t mn = __reduce_min_sync(peers, key), mx = __reduce_max_sync(peers, key);
-                        if (lane == __ffs(peers) - 1) { atomicMin(&okmin[sl], mn); atomicMax(&okmax[sl], mx); }
+                        if (lane == __ffs(peers) - 1) { atomicMin(&okmin[so], mn); atomicMax(&okmax[so], mx); }
                     } else {
                         const uint32_t pos = atomicAdd(&nbuf, 1u);
-                        buf_key[pos] = float_key(x);
+                        buf_key[pos] = float_key(x[j]);
                         buf_slot[pos] = (uint8_t)s;
                     }
                 }
@@ -564,7 +566,8 @@ __global__ void grid_init_kernel(Ctrl* ctrl, int mode, const float* T01_user) {
 }  // namespace
 
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
-                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st) {
+                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st,
+                        bool hist_done) {
     if (init != AAAC_INIT_QUANTILE) {
         grid_init_kernel<<<1, 32, 0, st>>>(ws.ctrl, mode, init == AAAC_INIT_USER ? T01_user : nullptr);
         note_launch();
@@ -587,10 +590,13 @@ cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, in
         rq.frac[e] = pos - lo;
     }
     cudaError_t e;
-    if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) return e;
     const int blocks = sm_count() * 3;
     const size_t sm0 = kQBins * sizeof(uint32_t);
-    if (mode == AAAC_INT4) {
+    if (hist_done) {
+        // the scales pass has already counted the histogram (launch_scales with with_hist)
+    } else if ((e = cudaMemsetAsync(ws.qhist, 0, kQBins * sizeof(uint32_t), st)) != cudaSuccess) {
+        return e;
+    } else if (mode == AAAC_INT4) {
         if ((e = cudaFuncSetAttribute(quantile_hist_kernel<AAAC_INT4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm0)) != cudaSuccess) return e;
         quantile_hist_kernel<AAAC_INT4><<<blocks, 512, sm0, st>>>(W, N, K, ldw, scales, ws.ctrl, ws.qhist);
         note_launch();

@@ -14,7 +14,7 @@ constexpr int kPartStride = 128;  // doubles per block partial (pack: [2][31] S,
 constexpr int kMaxBlocks = 2048;  // upper bound on fit-kernel grid size
 constexpr int kQBins = 16384;     // first-level histogram bins of the quantile selection
 constexpr int kQReq = 64;         // order statistics requested (2 per table entry)
-constexpr int kActMaxSplits = 256;
+constexpr int kActMaxSplits = 32;   // row strips of the activation statistics (the second kernel adds them one after the other)
 
 // shape of the fit-round kernel: warps per block, copies of the {J_low, thr} table
 #ifndef AAAC_FIT_WARPS
@@ -92,6 +92,13 @@ __device__ __forceinline__ uint32_t e4m3_encode(float x) {
     return u > 0x7Eu ? 0x7Eu : u;
 }
 
+// bin = floor(1024 x + 8192): one multiply-add rounded down onto 1.5 * 2^23 (where floats are
+// spaced by 1) leaves the integer in the low mantissa bits; the mask keeps any input inside the
+// table (|w~| < 8 by the scale rules, so for finite weights it changes nothing)
+__device__ __forceinline__ int qbin(float x) {
+    return (int)(__float_as_uint(__fmaf_rd(x, 1024.f, 8192.f + 12582912.f)) & (uint32_t)(kQBins - 1));
+}
+
 // Walks the items first, first + stride, first + 2 stride, ... of an N x slabs grid (row-major)
 // without a division per step; row runs past N when the walk is over.
 struct SlabWalk {
@@ -112,10 +119,13 @@ __device__ __forceinline__ float f32_round_down(double d) { return __double2floa
 // ---- launchers (each enqueues on `st` and returns the launch status) ----
 cudaError_t launch_act_stats(const uint16_t* X, int64_t T, int64_t K, int64_t ldx, float* I, int accumulate,
                              uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+// with_hist: the scales pass also counts the 16384-bin histogram of the normalised weights (the quantile
+// start's first pass over W) into ws.qhist; launch_init is then told so
 cudaError_t launch_scales(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, void* scales,
-                          float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+                          float* tensor_scale, uint32_t* dev_status, const Workspace& ws, cudaStream_t st, bool with_hist = false);
 cudaError_t launch_init(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int init,
-                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st);
+                        const void* scales, const float* T01_user, uint32_t* dev_status, const Workspace& ws, cudaStream_t st,
+                        bool hist_done = false);
 int act_splits_max(int64_t K);    // most row strips launch_act_stats uses for K input channels (sizes its partials)
 cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group, const void* scales,
                               const float* I, int n_outer, int n_inner, double* err_trace, float* T01_out, uint32_t* dev_status,
