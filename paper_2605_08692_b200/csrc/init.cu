@@ -270,24 +270,34 @@ quantile_plan_kernel(Ctrl* ctrl, const uint32_t* __restrict__ hist, uint8_t* __r
     }
     __syncthreads();
     {
-        // the requests whose rank lies in this thread's chunk (the last chunk also takes ranks beyond
-        // the data, which are never requested): walk the chunk's bins in registers
+        // The requests whose rank lies in this thread's chunk (the last chunk also takes ranks beyond the
+        // data, which are never requested).  A warp first sieves the 64 requests against the range of
+        // its 32 chunks, two requests per lane, and only the few that pass are looked at by every lane;
+        // the owning thread then walks its chunk's bins in registers.
         const unsigned long long lo = chunk[tid], hi = lo + s;
-        for (int q = 0; q < kQReq; ++q) {
-            const unsigned long long r = req_rank[q];
-            if (!(r >= lo && (r < hi || tid == 1023))) continue;
-            if (r >= hi && tid != 1023) continue;
-            unsigned long long base = lo;
-            int i = 0;
+        const int lane = tid & 31, warp = tid >> 5;
+        const unsigned long long wlo = __shfl_sync(0xFFFFFFFFu, lo, 0), whi = __shfl_sync(0xFFFFFFFFu, hi, 31);
 #pragma unroll
-            for (int k = 0; k < per - 1; ++k)
-                if (i == k && r >= base + h[k]) { base += h[k]; ++i; }
-            uint32_t hv = h[0];
+        for (int half = 0; half < kQReq / 32; ++half) {
+            const unsigned long long rq_ = req_rank[half * 32 + lane];
+            unsigned mask = __ballot_sync(0xFFFFFFFFu, rq_ >= wlo && (rq_ < whi || warp == 31));
+            while (mask) {
+                const int q = half * 32 + __ffs(mask) - 1;
+                mask &= mask - 1;
+                const unsigned long long r = req_rank[q];
+                if (!(r >= lo && (r < hi || tid == 1023))) continue;
+                unsigned long long base = lo;
+                int i = 0;
 #pragma unroll
-            for (int k = 1; k < per; ++k) if (i == k) hv = h[k];
-            req_bin[q] = tid * per + i;
-            req_cnt[q] = hv;
-            ctrl->req_local[q] = r - base;
+                for (int k = 0; k < per - 1; ++k)
+                    if (i == k && r >= base + h[k]) { base += h[k]; ++i; }
+                uint32_t hv = h[0];
+#pragma unroll
+                for (int k = 1; k < per; ++k) if (i == k) hv = h[k];
+                req_bin[q] = tid * per + i;
+                req_cnt[q] = hv;
+                ctrl->req_local[q] = r - base;
+            }
         }
     }
     __syncthreads();
