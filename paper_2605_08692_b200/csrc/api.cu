@@ -1,4 +1,5 @@
 // C ABI of the library: argument validation, workspace carving, launch sequencing.
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 
@@ -108,6 +109,37 @@ struct Timing {
     cudaEvent_t* ev = nullptr;      // 2 per launch
 } g_timing;
 
+// Side streams of one device.  The layers of a batch are independent until their common fit
+// launch, so their scales and start passes are queued on streams of their own, forked from the
+// caller's stream and joined back to it: the small latency-bound kernels of one layer (plan,
+// selection, the tails of the streaming passes) then run under the bandwidth-bound passes of another.
+constexpr int kSideStreams = 7;
+constexpr int kMaxDevices = 64;
+struct SideStreams {
+    bool tried = false, ok = false;
+    cudaStream_t s[kSideStreams];
+    cudaEvent_t fork, join[kSideStreams];
+};
+std::mutex g_side_mu;                  // held while a call queues work on the side streams
+SideStreams g_side[kMaxDevices];
+
+// the current device's side streams (created on first use), or nullptr: then everything stays on the caller's stream
+SideStreams* side_streams() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    SideStreams& p = g_side[dev];
+    if (!p.tried) {
+        p.tried = true;
+        bool ok = cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < kSideStreams && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&p.s[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.join[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        p.ok = ok;
+    }
+    return p.ok ? &p : nullptr;
+}
+
 }  // namespace
 }  // namespace aaac
 
@@ -214,12 +246,33 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     FitLayerArgs* args = new FitLayerArgs[(size_t)n_layers];
     int rc = AAAC_OK;
-    for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
-        const aaac_layer& L = layers[l];
-        const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
-        const float* I = nullptr;
-        rc = prepare_fit_layer(L, mode, init, dev_status, w, st, &I);
-        args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, L.T01, w};
+    {
+        // layer l is prepared on lane l mod (1 + side streams); lane 0 is the caller's stream
+        std::unique_lock<std::mutex> lk(g_side_mu, std::defer_lock);
+        SideStreams* side = nullptr;
+        if (n_layers > 1) {
+            lk.lock();
+            side = side_streams();
+        }
+        const int lanes = side ? std::min(n_layers, kSideStreams + 1) : 1;
+        if (lanes > 1) {
+            if (cudaEventRecord(side->fork, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
+            for (int i = 0; i + 1 < lanes && rc == AAAC_OK; ++i)
+                if (cudaStreamWaitEvent(side->s[i], side->fork, 0) != cudaSuccess) rc = AAAC_ERR_CUDA;
+        }
+        for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
+            const aaac_layer& L = layers[l];
+            const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
+            const float* I = nullptr;
+            const int lane = l % lanes;
+            rc = prepare_fit_layer(L, mode, init, dev_status, w, lane == 0 ? st : side->s[lane - 1], &I);
+            args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, L.T01, w};
+        }
+        // joined even after an error, so that no side stream is left outside the caller's stream's order
+        for (int i = 0; i + 1 < lanes; ++i)
+            if (cudaEventRecord(side->join[i], side->s[i]) != cudaSuccess ||
+                cudaStreamWaitEvent(st, side->join[i], 0) != cudaSuccess)
+                rc = AAAC_ERR_CUDA;
     }
     if (rc == AAAC_OK) {
         // all rounds run in one launch per batch; the optional timing brackets the launches of this call
