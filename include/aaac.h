@@ -220,7 +220,7 @@ int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* si
  * are computed per layer exactly as by aaac_fit_layer_sel.  With more than one layer these
  * per-layer passes are queued on up to seven streams the library keeps per device (created at the
  * first such call), forked from `stream` and joined back to it before the fit launch: seen from
- * `stream`, the call is ordered like any other, and it may be captured into a graph.
+ * `stream`, the call is ordered like any other.
  *
  *   layers   HOST array of n_layers descriptors (read before the call returns); every pointer
  *            inside is a DEVICE pointer with the meaning, layout and alignment of the

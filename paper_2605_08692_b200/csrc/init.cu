@@ -92,7 +92,7 @@ quantile_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64
 
 // Step 3: candidates of the slotted bins, staged per block.
 constexpr int kStageCap = 4096;                  // staged candidates per block
-constexpr int kStageRoom = 256 * 8;              // most candidates one block iteration can add
+constexpr int kStageEvery = 4;                   // loop iterations between two looks at the stage's fill
 
 template <int MODE>
 __global__ void __launch_bounds__(256)
@@ -121,10 +121,10 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + tid) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t iters = (items + nwarps - 1) / nwarps;
+    const int64_t iters = (items + 2 * nwarps - 1) / (2 * nwarps);     // two items per warp and iteration
 
-    auto flush = [&]() {                                  // called by the whole block
-        const uint32_t n = nbuf;
+    auto flush = [&]() {                                  // called by the whole block, after a barrier
+        const uint32_t n = min(nbuf, (uint32_t)kStageCap);
         if (tid < kQReq) cnt[tid] = 0;
         __syncthreads();
         for (uint32_t i = tid; i < n; i += blockDim.x) buf_pos[i] = (uint16_t)atomicAdd(&cnt[buf_slot[i]], 1u);
@@ -138,12 +138,7 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
         __syncthreads();
     };
 
-    // The load of iteration k + 1 is issued before iteration k is processed, so that the block
-    // barrier at the end of an iteration does not wait for memory.
     SlabWalk it(warp0, nwarps, slabs);
-    uint4 v = make_uint4(0, 0, 0, 0);
-    float r = 0.f;
-    bool ok = false;
     auto fetch = [&](uint4& vv, float& rr, bool& okk) {
         const int64_t row = it.row, col = (int64_t)it.slab * 256 + lane * 8;
         okk = row < N && col < K;
@@ -155,49 +150,70 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
         }
         it.next();
     };
-    fetch(v, r, ok);
-    for (int64_t k = 0; k < iters; ++k) {
-        uint4 vn;
-        float rn;
-        bool okn;
-        fetch(vn, rn, okn);
-        if (ok) {
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-            // the slots of the lane's eight weights first (most rows hold no candidate at all: one test)
-            float x[8];
-            uint32_t sl[8], all = 0xFFu;
+    // The slots of a lane's eight weights first.  A slot byte has bit 7 set where the bin is not asked
+    // for, so the AND of the eight bytes tells whether the lane holds a candidate; a lane that does
+    // walks only its candidates (one, nearly always), found by a bit scan of the packed bytes, and
+    // recomputes w~ of that weight alone.
+    auto take = [&](const uint4& v, float r) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t sl[8], all = 0x80u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r);
-                sl[j] = sm_slot[qbin(x[j])];
-                all &= sl[j];
-            }
-            if (all != 0xFFu) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t s = sl[j];
-                    if (s == 0xFFu) continue;
-                    if (s & kSlotOver) {
-                        // no list space for this slot: keep only the extremes of its keys (lanes with the
-                        // same slot combine first, so that a heavy bin costs one atomic per warp step)
-                        const uint32_t key = float_key(x[j]), so = s & (kSlotOver - 1u);
-                        const unsigned peers = __match_any_sync(__activemask(), so);
-                        const uint32_t mn = __reduce_min_sync(peers, key), mx = __reduce_max_sync(peers, key);
-                        if (lane == __ffs(peers) - 1) { atomicMin(&okmin[so], mn); atomicMax(&okmax[so], mx); }
-                    } else {
-                        const uint32_t pos = atomicAdd(&nbuf, 1u);
-                        buf_key[pos] = float_key(x[j]);
-                        buf_slot[pos] = (uint8_t)s;
-                    }
+        for (int j = 0; j < 8; ++j) {
+            sl[j] = sm_slot[qbin(__fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), r))];
+            all &= sl[j];
+        }
+        if (all) return;
+        const uint32_t lo = __byte_perm(__byte_perm(sl[0], sl[1], 0x0040), __byte_perm(sl[2], sl[3], 0x0040), 0x5410);
+        const uint32_t hi = __byte_perm(__byte_perm(sl[4], sl[5], 0x0040), __byte_perm(sl[6], sl[7], 0x0040), 0x5410);
+        const uint64_t bytes = ((uint64_t)hi << 32) | lo;
+        uint64_t todo = ~bytes & 0x8080808080808080ull;
+        while (todo) {
+            const int j = (__ffsll((long long)todo) - 1) >> 3;
+            todo &= todo - 1;
+            const uint32_t s = (uint32_t)(bytes >> (8 * j)) & 0xFFu;
+            const uint32_t ww = (j >> 1) == 0 ? w[0] : (j >> 1) == 1 ? w[1] : (j >> 1) == 2 ? w[2] : w[3];
+            const uint32_t key = float_key(__fmul_rn((j & 1) ? bf16_hi(ww) : bf16_lo(ww), r));
+            if (s & kSlotOver) {
+                // no list space for this slot: keep only the extremes of its keys (lanes with the
+                // same slot combine first, so that a heavy bin costs one atomic per warp step)
+                const uint32_t so = s & (kSlotOver - 1u);
+                const unsigned peers = __match_any_sync(__activemask(), so);
+                const uint32_t mn = __reduce_min_sync(peers, key), mx = __reduce_max_sync(peers, key);
+                if (lane == __ffs(peers) - 1) { atomicMin(&okmin[so], mn); atomicMax(&okmax[so], mx); }
+            } else {
+                const uint32_t pos = atomicAdd(&nbuf, 1u);
+                if (pos < (uint32_t)kStageCap) {
+                    buf_key[pos] = key;
+                    buf_slot[pos] = (uint8_t)s;
+                } else {
+                    // the stage is full until the block next looks at it: straight to the slot's list
+                    list[ctrl->slot_off[s] + atomicAdd(&ctrl->slot_fill[s], 1u)] = key;
                 }
             }
         }
-        __syncthreads();
-        if (nbuf > kStageCap - kStageRoom) flush();       // uniform: nbuf is read after the barrier
-        v = vn;
-        r = rn;
-        ok = okn;
+    };
+
+    // Two items per warp are in flight: the loads of iteration k + 1 are issued before iteration k
+    // is processed.  The warps of a block meet only every kStageEvery iterations, to empty the
+    // stage once it is half full (the vote makes the decision the same for every thread).
+    uint4 va, vb;
+    float ra, rb;
+    bool oka, okb;
+    fetch(va, ra, oka);
+    fetch(vb, rb, okb);
+    for (int64_t k = 0; k < iters; ++k) {
+        uint4 vna, vnb;
+        float rna, rnb;
+        bool okna, oknb;
+        fetch(vna, rna, okna);
+        fetch(vnb, rnb, oknb);
+        if (oka) take(va, ra);
+        if (okb) take(vb, rb);
+        if ((k % kStageEvery) == kStageEvery - 1 && __syncthreads_or(nbuf > (uint32_t)kStageCap / 2)) flush();
+        va = vna; ra = rna; oka = okna;
+        vb = vnb; rb = rnb; okb = oknb;
     }
+    __syncthreads();
     flush();
     if (tid < kQReq && okmin[tid] <= okmax[tid]) {
         atomicMin(&ctrl->slot_kmin[tid], okmin[tid]);
