@@ -195,7 +195,7 @@ def run_reference(args, rank):
 
 CFG2_WORKLOAD = ("cfg2: Llama-3-8B-shaped q_proj 4096x4096, gate_proj 14336x4096, down_proj 4096x14336; NVFP4 g16 E4M3 "
                  "scales; X 4096 tokens; quantile init; 20 rounds; step = act_stats + scales + init + 20 fit rounds + "
-                 "pack + dequant per layer")
+                 "pack + dequant of the three layers (one aaac_quantize_layers call)")
 
 STACKS = {
     # name: (decoder layers, hidden, kv width, intermediate, mode, tokens, rounds)
@@ -256,20 +256,17 @@ def run_stack(args, which, emit=True):
     Iv = {k: torch.empty(x.shape[1], dtype=torch.float32, device=dev) for k, x in X.items()}
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    descs = [dict(W=Ws[n], I=Iv[xin], T01=out[n]["T01"], scales=out[n]["scales"], tensor_scale=out[n]["ts"], ws=out[n]["ws"])
+    descs = [dict(W=Ws[n], I=Iv[xin], T01=out[n]["T01"], scales=out[n]["scales"], tensor_scale=out[n]["ts"], ws=out[n]["ws"],
+                  T01_bf16=out[n]["Tb"], codes=out[n]["codes"], err_out=out[n]["err"], sigma_bits=out[n]["bits"])
              for n, N, K, xin in lin]
 
     def decoder_layer():
         for k, x in X.items():
             binding.act_stats(x, Iv[k], out["down" if k == "down" else "q"]["ws"], dev_status=status)
-        # the seven linears of a decoder layer are independent: one aaac_fit_layers call
-        binding.fit_layers(descs, mode, n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE, dev_status=status,
-                           sel_group=sel)
-        for n, N, K, xin in lin:
-            o = out[n]
-            binding.pack(Ws[n], mode, I=Iv[xin], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"],
-                         tensor_scale=o["ts"], codes=o["codes"], ws=o["ws"], err_out=o["err"], sel_group=sel,
-                         sigma_bits=o["bits"])
+        # the seven linears of a decoder layer are independent: one aaac_quantize_layers call (scales, start,
+        # rounds in one launch, pack)
+        binding.quantize_layers(descs, mode, n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE, dev_status=status,
+                                sel_group=sel)
 
     for _ in range(2):
         decoder_layer()
@@ -295,8 +292,8 @@ def run_stack(args, which, emit=True):
             "dtype": "f32", "data": "synthetic (device-generated, one decoder layer's tensors reused for every layer)",
             "config": {"workload": f"{which}: {L} decoder layers x 7 linears (hidden {H}, kv {KV}, intermediate {FF}), "
                                    f"{'INT4 g128' if mode == 0 else 'NVFP4 g16'} S{sel or g}, {tokens} tokens per input, quantile init, "
-                                   f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds (the seven linears of a "
-                                   f"decoder layer in one aaac_fit_layers call) + pack",
+                                   f"n_outer {rounds}, n_inner {n_inner}; act_stats + scales + init + rounds + pack (the seven linears of a "
+                                   f"decoder layer in one aaac_quantize_layers call)",
                        "linears": 7 * L, "weights": wl * L, "rounds": rounds, "n_inner": n_inner},
             "gweights_per_s_per_round": wl * L * rounds * n_inner / wall / 1e9, "clocks": clocks,
             "gpu_launches": launches_per_layer * L}
@@ -393,22 +390,22 @@ def main():
             ws=binding.alloc_workspace(mode, N, K, TOKENS, dev)))
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    descs = [dict(W=W, I=o["I"], T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"]) for W, o in zip(Wd, outs)]
+    descs = [dict(W=W, X=X, T01=o["T01"], scales=o["scales"], tensor_scale=o["ts"], ws=o["ws"], T01_bf16=o["Tb"],
+                  codes=o["codes"], err_out=o["err"], What=o["What"]) for W, X, o in zip(Wd, Xd, outs)]
+    descs_I = [dict(d, X=None, I=o["I"]) for d, o in zip(descs, outs)]
     ones = {K: torch.ones(K, dtype=torch.float32, device=dev) for _, K in shapes} if args.with_prescale else {}
 
     def step():
-        # the layers of a step are independent: their importances first, then scales, start tables and the
-        # 20 rounds of all of them in one aaac_fit_layers call (the rounds in one launch), then pack and dequant
-        for X, o in zip(Xd, outs):
-            binding.act_stats(X, o["I"], o["ws"], dev_status=status)
+        # the layers of a step are independent problems: one aaac_quantize_layers call takes them through the
+        # whole path (importances from X, scales, start tables, the 20 rounds of all of them in one launch,
+        # pack, reconstruction)
         if args.with_prescale:
-            for W, o in zip(Wd, outs):
+            for X, W, o in zip(Xd, Wd, outs):
+                binding.act_stats(X, o["I"], o["ws"], dev_status=status)
                 binding.prescale_columns(W, ones[W.shape[1]], o["What"], o["I"], o["I"], dev_status=status)
-        binding.fit_layers(descs, mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE, dev_status=status)
-        for W, o in zip(Wd, outs):
-            binding.pack(W, mode, I=o["I"], T01=o["T01"], T01_bf16=o["Tb"], scales=o["scales"], tensor_scale=o["ts"],
-                         codes=o["codes"], ws=o["ws"], err_out=o["err"])
-            binding.dequant(o["codes"], o["scales"], o["ts"], o["Tb"], mode, o["What"])
+            binding.quantize_layers(descs_I, mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE, dev_status=status)
+            return
+        binding.quantize_layers(descs, mode, n_outer=ROUNDS, init=binding.INIT_QUANTILE, dev_status=status)
 
     def barrier():
         if world > 1:

@@ -246,6 +246,39 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
                     int n_outer, int n_inner, int init, uint32_t* dev_status /* may be NULL */, void* stream);
 
 /*
+ * The whole path of Algorithm 1 for several layers in one call: aaac_fit_layers on the batch,
+ * then for every layer the pack pass (Eq. 6, Eq. 8) and, where `What` is given, the
+ * dequantisation (Eq. 5).  The results are those of the separate calls on each layer; the
+ * per-layer passes before and after the fit launch are queued on the library's side streams
+ * (see aaac_fit_layers), forked from `stream` and joined back to it.
+ *
+ *   layers   as for aaac_fit_layers (the pack pass uses the importance the fit used: I, or
+ *            the one computed from X, which stays in the layer's ws)
+ *   outs     HOST array of n_layers descriptors, DEVICE pointers inside:
+ *              T01_bf16   [2][16] BF16 bit patterns, written (the tables as stored, Sec. 3.2)
+ *              codes      [N][K/2] packed 4-bit codes, written; 16-byte aligned
+ *              sigma_bits [N][K/128] selection bytes, written; only where sel_group != group, else ignored
+ *              err_out    [2] doubles: Eq. 2 objective with the stored tables, sum of w^2 I; or NULL
+ *              stats      [4] counters of aaac_pack; or NULL
+ *              What       [N][ldo] BF16 reconstruction, written; or NULL: no dequantisation
+ *              ldo        elements between rows of What (>= K, multiple of 8)
+ * Returns the first error found (nothing is enqueued for an invalid batch).
+ */
+typedef struct {
+    uint16_t* T01_bf16;
+    uint8_t* codes;
+    uint8_t* sigma_bits;
+    double* err_out;
+    uint64_t* stats;
+    void* What;
+    int64_t ldo;
+} aaac_layer_out;
+
+int aaac_quantize_layers(const aaac_layer* layers, const aaac_layer_out* outs, int n_layers, int mode, int group,
+                         int sel_group, int n_outer, int n_inner, int init, uint32_t* dev_status /* may be NULL */,
+                         void* stream);
+
+/*
  * Per-input-channel scaling before the fit (Section 4, "Combining AAAC with AWQ": AWQ scales
  * the weights, AAAC then learns its tables on the scaled distribution).  The multipliers a_k
  * themselves come from the caller (AWQ's search is not part of the method).

@@ -24,7 +24,8 @@ _lib = None
 EXPORTS = ["aaac_status_string", "aaac_workspace_bytes", "aaac_act_stats", "aaac_fit_layer", "aaac_pack",
            "aaac_dequant", "aaac_act_stats_noalloc", "aaac_host_workspace_bytes", "aaac_quantize_layer_host", "aaac_timing_begin",
            "aaac_timing_end", "aaac_fit_layer_sel", "aaac_pack_sel", "aaac_dequant_sel", "aaac_prescale_columns",
-           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait", "aaac_fit_layers", "aaac_workspace_bytes_full", "aaac_debug_quantile_cap"]
+           "aaac_quantize_layer_host_async", "aaac_launch_count", "aaac_debug_fit_wait", "aaac_fit_layers", "aaac_workspace_bytes_full", "aaac_debug_quantile_cap",
+           "aaac_quantize_layers"]
 
 
 class AaacError(RuntimeError):
@@ -75,6 +76,8 @@ def lib():
         L.aaac_quantize_layer_host_async.restype = ci
         L.aaac_fit_layers.argtypes = [C.POINTER(LayerDesc), ci, ci, ci, ci, ci, ci, ci, vp, vp]
         L.aaac_fit_layers.restype = ci
+        L.aaac_quantize_layers.argtypes = [C.POINTER(LayerDesc), C.POINTER(LayerOut), ci, ci, ci, ci, ci, ci, ci, vp, vp]
+        L.aaac_quantize_layers.restype = ci
         L.aaac_debug_quantile_cap.argtypes = [C.c_size_t]
         L.aaac_debug_quantile_cap.restype = ci
         L.aaac_debug_fit_wait.argtypes = [ci, C.c_uint]
@@ -155,6 +158,18 @@ def fit_layers(layers, mode, *, n_outer, init, n_inner=1, group=None, sel_group=
     """aaac_fit_layers: `layers` is a list of dicts with the keyword arguments of fit_layer that belong
     to one layer (W, I or X, T01, scales, tensor_scale, ws, optionally err_trace)."""
     g = group or group_of(mode)
+    arr = _layer_descs(layers)
+    _check(lib().aaac_fit_layers(arr, len(layers), mode, g, sel_group or g, n_outer, n_inner, init, _ptr(dev_status),
+                                 _stream()))
+
+
+class LayerOut(C.Structure):
+    """aaac_layer_out of include/aaac.h."""
+    _fields_ = [("T01_bf16", C.c_void_p), ("codes", C.c_void_p), ("sigma_bits", C.c_void_p), ("err_out", C.c_void_p),
+                ("stats", C.c_void_p), ("What", C.c_void_p), ("ldo", C.c_int64)]
+
+
+def _layer_descs(layers):
     arr = (LayerDesc * len(layers))()
     for d, a in zip(arr, layers):
         W, X = a["W"], a.get("X")
@@ -165,8 +180,23 @@ def fit_layers(layers, mode, *, n_outer, init, n_inner=1, group=None, sel_group=
         d.T01, d.scales, d.tensor_scale = a["T01"].data_ptr(), a["scales"].data_ptr(), a["tensor_scale"].data_ptr()
         d.err_trace = a["err_trace"].data_ptr() if a.get("err_trace") is not None else None
         d.ws, d.ws_bytes = a["ws"].data_ptr(), a["ws"].numel()
-    _check(lib().aaac_fit_layers(arr, len(layers), mode, g, sel_group or g, n_outer, n_inner, init, _ptr(dev_status),
-                                 _stream()))
+    return arr
+
+
+def quantize_layers(layers, mode, *, n_outer, init, n_inner=1, group=None, sel_group=None, dev_status=None):
+    """aaac_quantize_layers: the dicts of fit_layers plus the outputs of the pack pass (T01_bf16, codes,
+    optionally sigma_bits, err_out, stats) and optionally What for the reconstruction."""
+    g = group or group_of(mode)
+    arr = _layer_descs(layers)
+    outs = (LayerOut * len(layers))()
+    for o, a in zip(outs, layers):
+        o.T01_bf16, o.codes = a["T01_bf16"].data_ptr(), a["codes"].data_ptr()
+        for name in ("sigma_bits", "err_out", "stats"):
+            setattr(o, name, a[name].data_ptr() if a.get(name) is not None else None)
+        What = a.get("What")
+        o.What, o.ldo = (What.data_ptr(), What.stride(0)) if What is not None else (None, 0)
+    _check(lib().aaac_quantize_layers(arr, outs, len(layers), mode, g, sel_group or g, n_outer, n_inner, init,
+                                      _ptr(dev_status), _stream()))
 
 
 def pack(W, mode, *, I, T01, T01_bf16, scales, tensor_scale, codes, ws, err_out=None, stats=None, group=None,

@@ -140,6 +140,44 @@ SideStreams* side_streams() {
     return p.ok ? &p : nullptr;
 }
 
+// Lanes for n independent pieces of work: lane 0 is the caller's stream, the others are side
+// streams that wait for what the caller's stream holds so far; join() makes the caller's stream
+// wait for all of them again.  One lane (no side streams, or n = 1) is the caller's stream alone.
+class Lanes {
+public:
+    Lanes(cudaStream_t st, int n) : lk_(g_side_mu, std::defer_lock), st_(st) {
+        if (n > 1) {
+            lk_.lock();
+            side_ = side_streams();
+        }
+        lanes_ = side_ ? std::min(n, kSideStreams + 1) : 1;
+        if (lanes_ > 1) {
+            ok_ = cudaEventRecord(side_->fork, st_) == cudaSuccess;
+            for (int i = 0; i + 1 < lanes_ && ok_; ++i) ok_ = cudaStreamWaitEvent(side_->s[i], side_->fork, 0) == cudaSuccess;
+        }
+    }
+    bool ok() const { return ok_; }
+    cudaStream_t of(int l) const {
+        const int lane = l % lanes_;
+        return lane == 0 ? st_ : side_->s[lane - 1];
+    }
+    // always called, also after an error, so that no side stream is left outside the caller's stream's order
+    bool join() {
+        for (int i = 0; i + 1 < lanes_; ++i)
+            if (cudaEventRecord(side_->join[i], side_->s[i]) != cudaSuccess ||
+                cudaStreamWaitEvent(st_, side_->join[i], 0) != cudaSuccess)
+                ok_ = false;
+        lanes_ = 1;
+        return ok_;
+    }
+private:
+    std::unique_lock<std::mutex> lk_;
+    SideStreams* side_ = nullptr;
+    cudaStream_t st_;
+    int lanes_ = 1;
+    bool ok_ = true;
+};
+
 }  // namespace
 }  // namespace aaac
 
@@ -247,32 +285,16 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
     FitLayerArgs* args = new FitLayerArgs[(size_t)n_layers];
     int rc = AAAC_OK;
     {
-        // layer l is prepared on lane l mod (1 + side streams); lane 0 is the caller's stream
-        std::unique_lock<std::mutex> lk(g_side_mu, std::defer_lock);
-        SideStreams* side = nullptr;
-        if (n_layers > 1) {
-            lk.lock();
-            side = side_streams();
-        }
-        const int lanes = side ? std::min(n_layers, kSideStreams + 1) : 1;
-        if (lanes > 1) {
-            if (cudaEventRecord(side->fork, st) != cudaSuccess) rc = AAAC_ERR_CUDA;
-            for (int i = 0; i + 1 < lanes && rc == AAAC_OK; ++i)
-                if (cudaStreamWaitEvent(side->s[i], side->fork, 0) != cudaSuccess) rc = AAAC_ERR_CUDA;
-        }
+        Lanes lanes(st, n_layers);
+        if (!lanes.ok()) rc = AAAC_ERR_CUDA;
         for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
             const aaac_layer& L = layers[l];
             const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
             const float* I = nullptr;
-            const int lane = l % lanes;
-            rc = prepare_fit_layer(L, mode, init, dev_status, w, lane == 0 ? st : side->s[lane - 1], &I);
+            rc = prepare_fit_layer(L, mode, init, dev_status, w, lanes.of(l), &I);
             args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, L.T01, w};
         }
-        // joined even after an error, so that no side stream is left outside the caller's stream's order
-        for (int i = 0; i + 1 < lanes; ++i)
-            if (cudaEventRecord(side->join[i], side->s[i]) != cudaSuccess ||
-                cudaStreamWaitEvent(st, side->join[i], 0) != cudaSuccess)
-                rc = AAAC_ERR_CUDA;
+        if (!lanes.join() && rc == AAAC_OK) rc = AAAC_ERR_CUDA;
     }
     if (rc == AAAC_OK) {
         // all rounds run in one launch per batch; the optional timing brackets the launches of this call
@@ -305,6 +327,24 @@ int aaac_fit_layer_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mod
     return aaac_fit_layers(&L, 1, mode, group, sel_group, n_outer, n_inner, init, dev_status, stream);
 }
 
+namespace {
+// the pack pass of one layer on `st`; arguments already checked
+int enqueue_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int sel_group,
+                 const float* I, const float* T01_f32, uint16_t* T01_bf16,
+                 void* scales, const float* tensor_scale, uint8_t* codes, uint8_t* sigma_bits,
+                 double* err_out, uint64_t* stats, void* ws, size_t ws_bytes, cudaStream_t stream) {
+    Workspace w = carve(ws, mode, N, K, ws_bytes);
+    cudaStream_t st = stream;
+    // the pack pass uses only the block counter and its own result fields of the control block
+    if (cudaMemsetAsync(&w.ctrl->done, 0, sizeof(uint32_t), st) != cudaSuccess) return AAAC_ERR_CUDA;
+    if (cudaMemsetAsync(w.ctrl->pack_err, 0, sizeof(double) * 2 + sizeof(unsigned long long) * 4, st) != cudaSuccess)
+        return AAAC_ERR_CUDA;
+    return launch_pack(static_cast<const uint16_t*>(W), N, K, ldw, mode, sel_group, I, T01_f32, T01_bf16, scales,
+                       tensor_scale, codes, sigma_bits, err_out, reinterpret_cast<unsigned long long*>(stats), w, st) == cudaSuccess
+               ? AAAC_OK : AAAC_ERR_CUDA;
+}
+}  // namespace
+
 int aaac_pack(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, int group,
               const float* I, const float* T01_f32, uint16_t* T01_bf16,
               void* scales, const float* tensor_scale, uint8_t* codes,
@@ -327,15 +367,45 @@ int aaac_pack_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, in
     if (!aligned(I, 16) || !aligned(codes, 16) || !aligned(T01_bf16, 2)) return AAAC_ERR_ALIGN;
     rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
     if (rc) return rc;
-    Workspace w = carve(ws, mode, N, K, ws_bytes);
+    return enqueue_pack(W, N, K, ldw, mode, sel_group, I, T01_f32, T01_bf16, scales, tensor_scale, codes, sigma_bits,
+                        err_out, stats, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int aaac_quantize_layers(const aaac_layer* layers, const aaac_layer_out* outs, int n_layers, int mode, int group,
+                         int sel_group, int n_outer, int n_inner, int init, uint32_t* dev_status, void* stream) {
+    if (!layers || !outs) return AAAC_ERR_NULL;
+    if (n_layers < 1 || n_layers > 4096) return AAAC_ERR_SHAPE;
+    for (int l = 0; l < n_layers; ++l) {
+        const aaac_layer& L = layers[l];
+        const aaac_layer_out& O = outs[l];
+        const int rc = check_fit_layer(L, mode, group, sel_group, n_outer, n_inner, init);
+        if (rc) return rc;
+        if (!O.T01_bf16 || !O.codes) return AAAC_ERR_NULL;
+        if (sel_group != group && !O.sigma_bits) return AAAC_ERR_NULL;
+        if (!aligned(O.codes, 16) || !aligned(O.T01_bf16, 2)) return AAAC_ERR_ALIGN;
+        if (O.What && (O.ldo < L.K || O.ldo % 8)) return AAAC_ERR_SHAPE;
+        if (O.What && !aligned(O.What, 16)) return AAAC_ERR_ALIGN;
+    }
+    int rc = aaac_fit_layers(layers, n_layers, mode, group, sel_group, n_outer, n_inner, init, dev_status, stream);
+    if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the pack pass uses only the block counter and its own result fields of the control block
-    if (cudaMemsetAsync(&w.ctrl->done, 0, sizeof(uint32_t), st) != cudaSuccess) return AAAC_ERR_CUDA;
-    if (cudaMemsetAsync(w.ctrl->pack_err, 0, sizeof(double) * 2 + sizeof(unsigned long long) * 4, st) != cudaSuccess)
-        return AAAC_ERR_CUDA;
-    return launch_pack(static_cast<const uint16_t*>(W), N, K, ldw, mode, sel_group, I, T01_f32, T01_bf16, scales,
-                       tensor_scale, codes, sigma_bits, err_out, reinterpret_cast<unsigned long long*>(stats), w, st) == cudaSuccess
-               ? AAAC_OK : AAAC_ERR_CUDA;
+    Lanes lanes(st, n_layers);
+    if (!lanes.ok()) rc = AAAC_ERR_CUDA;
+    for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
+        const aaac_layer& L = layers[l];
+        const aaac_layer_out& O = outs[l];
+        // the importance the fit used: the caller's, or the one the fit computed from X into the workspace
+        const float* I = L.I ? L.I : carve(L.ws, mode, L.N, L.K, L.ws_bytes).I;
+        uint8_t* sg = sel_group == group ? nullptr : O.sigma_bits;
+        rc = enqueue_pack(L.W, L.N, L.K, L.ldw, mode, sel_group, I, L.T01, O.T01_bf16, L.scales, L.tensor_scale, O.codes, sg,
+                          O.err_out, O.stats, L.ws, L.ws_bytes, lanes.of(l));
+        if (rc == AAAC_OK && O.What &&
+            launch_dequant(O.codes, L.scales, sg, L.tensor_scale, O.T01_bf16, L.N, L.K, mode, static_cast<uint16_t*>(O.What),
+                           O.ldo, lanes.of(l)) != cudaSuccess)
+            rc = AAAC_ERR_CUDA;
+    }
+    if (!lanes.join() && rc == AAAC_OK) rc = AAAC_ERR_CUDA;
+    return rc;
 }
 
 int aaac_dequant(const uint8_t* codes, const void* scales, const float* tensor_scale,

@@ -492,6 +492,81 @@ def test_fit_layers_more_layers_than_one_launch_takes_and_inner_refinement():
         assert np.allclose(host(d["err_trace"])[:2], o["trace"], rtol=1e-4)
 
 
+def run_quantize_batch(cases, mode, rounds, init, sel_group=None, what_pad=0):
+    """aaac_quantize_layers on a list of (W, X) cases, importances from X inside the call."""
+    g = 128 if mode == INT4 else 16
+    descs = []
+    for W, X in cases:
+        N, K = W.shape
+        d = dict(W=dev_bf16(W), X=dev_bf16(X),
+                 T01=torch.zeros(2, 16, dtype=torch.float32, device=DEV),
+                 scales=torch.empty(N, K // g, dtype=torch.uint16 if mode == INT4 else torch.uint8, device=DEV),
+                 tensor_scale=torch.ones(1, dtype=torch.float32, device=DEV),
+                 err_trace=torch.zeros(max(rounds, 1), dtype=torch.float64, device=DEV),
+                 ws=binding.alloc_workspace(mode, N, K, X.shape[0]),
+                 T01_bf16=torch.empty(2, 16, dtype=torch.uint16, device=DEV),
+                 codes=torch.empty(N, K // 2, dtype=torch.uint8, device=DEV),
+                 err_out=torch.zeros(2, dtype=torch.float64, device=DEV),
+                 stats=torch.zeros(4, dtype=torch.int64, device=DEV),
+                 What_full=torch.full((N, K + what_pad), 7.0, dtype=torch.bfloat16, device=DEV))
+        d["What"] = d["What_full"][:, :K]
+        if sel_group is not None:
+            d["sigma_bits"] = torch.zeros(N, K // (8 * sel_group), dtype=torch.uint8, device=DEV)
+        descs.append(d)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.quantize_layers(descs, mode, n_outer=rounds, init=init, sel_group=sel_group, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return descs
+
+
+@pytest.mark.parametrize("mode,sel", [(NVFP4, None), (INT4, None), (INT4, 16)])
+def test_quantize_layers_whole_path_matches_oracle_per_layer(mode, sel):
+    """The whole path for several layers in one call (importances from X, scales, start, rounds, pack,
+    reconstruction), more layers than there are side streams: every output of every layer against the oracle."""
+    g = 128 if mode == INT4 else 16
+    shapes = [(257, 1024), (3, 256), (70, 640), (1, 128), (300, 768), (40, 512), (64, 256), (9, 384), (129, 256)]
+    cases, oracles = [], []
+    for i, (N, K) in enumerate(shapes):
+        W, X = layer(mode, N, K, name=f"qbatch{mode}{sel}/{i}")
+        kw = dict(S=sel) if sel else {}
+        oracles.append(oracle.fit_layer(W, mode, g, 5, X=X, init="quantile", **kw))
+        cases.append((W, X))
+    a = run_quantize_batch(cases, mode, 5, binding.INIT_QUANTILE, sel_group=sel, what_pad=8)
+    b = run_quantize_batch(cases, mode, 5, binding.INIT_QUANTILE, sel_group=sel)
+    for i, (d, d2, o) in enumerate(zip(a, b, oracles)):
+        label = f"quantize_layers mode {mode} S {sel} layer {i}"
+        ok, worst = table_close(host(d["T01"]), o["T"])
+        assert ok, f"{label}: tables differ: worst {worst:.3e}"
+        assert np.allclose(host(d["err_trace"])[:5], o["trace"], rtol=1e-4, atol=0)
+        check_end_to_end_bits(d, o, label, sel=bool(sel))
+        assert np.isclose(host(d["err_out"])[0], o["E_final"], rtol=1e-4)
+        st = host(d["stats"])
+        assert st[0] == o["ties"][0] and st[1] == o["ties"][1]
+        if sel:
+            want = oracle.dequant_sel(o["codes"], o["scales"], o["tensor_scale"], o["T_bf16"], o["sigma_bits"], sel, mode, g)
+        else:
+            want = oracle.dequant(o["codes"], o["scales"], o["tensor_scale"], o["T_bf16"], mode, g)
+        assert np.array_equal(host(d["What"].contiguous()), want), f"{label}: reconstruction differs"
+        for k in ("T01", "T01_bf16", "codes", "scales", "err_out"):
+            assert torch.equal(d[k], d2[k]), f"{label}: {k} differs between two calls"
+        assert torch.equal(d["What"], d2["What"])
+        assert bool((d["What_full"][:, o["codes"].shape[1] * 2:] == 7.0).all()), f"{label}: wrote past a row of What"
+
+
+def test_quantize_layers_rejects_a_bad_output_before_enqueuing_anything():
+    W, X = layer(NVFP4, 16, 256, name="qbatchbad")
+    good = dict(W=dev_bf16(W), I=torch.ones(256, device=DEV), T01=torch.zeros(2, 16, device=DEV),
+                scales=torch.empty(16, 16, dtype=torch.uint8, device=DEV), tensor_scale=torch.ones(1, device=DEV),
+                ws=binding.alloc_workspace(NVFP4, 16, 256), T01_bf16=torch.empty(2, 16, dtype=torch.uint16, device=DEV),
+                codes=torch.empty(16, 128, dtype=torch.uint8, device=DEV))
+    bad = dict(good, What=torch.empty(16, 260, dtype=torch.bfloat16, device=DEV)[:, :256])      # row stride not a multiple of 8
+    before = binding.launch_count()
+    with pytest.raises(binding.AaacError, match="status"):
+        binding.quantize_layers([good, bad], NVFP4, n_outer=2, init=binding.INIT_GRID)
+    assert binding.launch_count() == before
+
+
 def test_fit_layers_rejects_a_bad_layer_before_enqueuing_anything():
     W, X = layer(NVFP4, 16, 256, name="batchbad")
     good = dict(W=dev_bf16(W), I=torch.ones(256, device=DEV), T01=torch.zeros(2, 16, device=DEV),
