@@ -261,7 +261,7 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
     // 32-bit shared addresses.  Slot offsets carry the address of this lane's column of the
     // {P, Q} table, so a lookup there needs no further arithmetic.
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
-    const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;                       // + bin * REP * 8
+    const uint32_t lut1_copy = (lane & (REP - 1)) * 8;                                 // this lane's copy of a bin's entry; | bin * REP * 8
     const uint32_t lut2_addr = sm_base + kLut1Bytes;                                   // the {P, Q} table
     const uint32_t bins_warp = sm_base + kLut1Bytes + kLut2Bytes + warp * kBinBytes;
     const uint32_t bins_lane = bins_warp + lane * 8;                                   // + cell * 256
@@ -429,8 +429,10 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask;
-                e1v[j] = lds_table_u2(lut1_lane + off);
+                // (bin bits | lane's copy) is one three-input logic instruction, and the table's base, the
+                // same for every lane, can ride in the load's address: no add per weight
+                const uint32_t off = ((uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask) | lut1_copy;
+                e1v[j] = lds_table_u2(sm_base + off);
             }
         };
         // same, then refill the row's registers from the next item

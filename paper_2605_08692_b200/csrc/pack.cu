@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
     build_tables<MODE, NW, REP, NB>(S, dyn);
 
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
-    const uint32_t lut1_lane = sm_base + (lane & (REP - 1)) * 8;
+    const uint32_t lut1_copy = (lane & (REP - 1)) * 8;             // this lane's copy of a bin's entry
     const uint32_t lut2_addr = sm_base + kLut1Bytes;                // the {P, Q} table
     constexpr float kBinsPerUnit = (float)(NB / 16);
     constexpr float kMagic = (float)(NB / 2) + 1.5f * (float)(1 << 23) / (float)(REP * 8);
@@ -228,8 +228,8 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
-                const uint32_t off = (uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask;
-                const uint2 e = lds_table_u2(lut1_lane + off);
+                const uint32_t off = ((uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask) | lut1_copy;
+                const uint2 e = lds_table_u2(sm_base + off);
                 tcand |= (x[j] == __uint_as_float(e.y));
                 pq[j] = lds_table_b64(above_addr(e.x, x[j], e.y));
                 const uint64_t u01 = diff2(x[j], pq[j]);
