@@ -52,7 +52,7 @@ typedef enum {
     AAAC_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed */
     AAAC_ERR_NONFINITE = 7,     /* (dev_status bit) W or X holds Inf / NaN */
     AAAC_ERR_UNIMPLEMENTED = 8, /* reserved */
-    AAAC_ERR_TOO_LARGE = 9,     /* size beyond the fixed capacity of a no-allocation entry point */
+    AAAC_ERR_TOO_LARGE = 9,     /* size beyond a fixed capacity: K of a no-allocation entry point, N * ldw of a fit */
     AAAC_ERR_TIMEOUT = 10       /* (dev_status bit AAAC_DEV_TIMEOUT) a bounded device-side wait ran out */
 } aaac_status;
 
@@ -131,7 +131,8 @@ int aaac_act_stats_noalloc(const void* X, int64_t T, int64_t K, int64_t ldx, flo
  * before the iteration, an entry whose cell has no weight keeping its value; sort }.  With
  * n_inner = 1 a round is a single pass over W (the cells of the update are the nearest-entry
  * indices of the assignment step); every further inner iteration is one more, cheaper pass.
- * n_inner >= 1 and n_outer * n_inner <= 2^20, else AAAC_ERR_SHAPE.
+ * n_inner >= 1 and n_outer * n_inner <= 2^20, else AAAC_ERR_SHAPE.  A layer must span fewer than
+ * 2^32 elements (N * ldw < 2^32; the fit kernels index it with 32 bits), else AAAC_ERR_TOO_LARGE.
  *
  *   scales        out  positive scales (sign bit clear).  INT4: s = bf16(absmax/7) (1 for an
  *                      all-zero group).  NVFP4: E4M3(absmax / (6 s_t)) in 0x01..0x7E with

@@ -244,6 +244,8 @@ int check_fit_layer(const aaac_layer& L, int mode, int group, int sel_group, int
     if (!sel_ok(mode, group, sel_group)) return AAAC_ERR_MODE;
     if (!L.T01 || !L.scales || !L.tensor_scale) return AAAC_ERR_NULL;
     if (!L.I && !L.X) return AAAC_ERR_NULL;
+    // the fit kernels index a layer's elements with 32 bits
+    if ((unsigned long long)L.N * (unsigned long long)L.ldw >= (1ull << 32)) return AAAC_ERR_TOO_LARGE;
     if (init != AAAC_INIT_QUANTILE && init != AAAC_INIT_GRID && init != AAAC_INIT_USER) return AAAC_ERR_MODE;
     if (n_outer < 0) return AAAC_ERR_SHAPE;
     if (n_inner < 1 || (int64_t)n_outer * n_inner > (1 << 20)) return AAAC_ERR_SHAPE;

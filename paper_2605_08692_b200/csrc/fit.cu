@@ -96,17 +96,6 @@ struct FitParams {
     int tail_item0, tail_quarters;   // items from tail_item0 on are dealt out a quarter (one row per warp) per block
 };
 
-// hi + lo += v, error-free (Knuth's two-sum in FP32; the intrinsics keep the compiler from
-// re-associating).  Double-precision arithmetic is slow on this GPU, so the in-kernel
-// reductions carry their sums as FP32 pairs and convert once at the end.
-__device__ __forceinline__ void two_sum(float& hi, float& lo, float v) {
-    const float s = __fadd_rn(hi, v);
-    const float bb = __fsub_rn(s, hi);
-    const float err = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(v, bb));
-    hi = s;
-    lo = __fadd_rn(lo, err);
-}
-
 constexpr int kMaxFitBlocks = 1024;                   // grid limit: block sums are added as 32-bit limbs, the arrivals counted in 16 bits
 constexpr int kLimbs = 3;                             // a sum is a 96-bit two's-complement fixed-point number
 constexpr unsigned kDefaultSpinLimit = 1u << 23;      // polls of >= 32 ns each: several seconds
@@ -350,8 +339,9 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
         sc[u] = 0u;
         if (INNER) sgw[u] = 0u;
         if (col0 < K && row < N) {
-            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
-            const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
+            // element offsets fit 32 bits (the entry points refuse layers of 2^32 elements and more)
+            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + ((unsigned)row * (unsigned)p.ldw + (unsigned)col0)));
+            const unsigned gi = (unsigned)row * (unsigned)Gr + (unsigned)col0 / G;
             if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];          // masked at use: nothing waits on the load here
             else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
             if (INNER) sgw[u] = __ldcg(p.sigw + (size_t)row * (size_t)slabs + slab);
@@ -591,18 +581,17 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
     //      rotated, fixed order that avoids bank conflicts); then the warps are added ----
     __syncthreads();                                       // every warp is done with the lookup tables
     {
-        // four interleaved error-free chains (the additions of one chain depend on each other)
-        float hx[4] = {0.f, 0.f, 0.f, 0.f}, lx[4] = {0.f, 0.f, 0.f, 0.f}, hy[4] = {0.f, 0.f, 0.f, 0.f}, ly[4] = {0.f, 0.f, 0.f, 0.f};
+        // four interleaved chains in double: 32 FP32 values go into 53 bits without rounding unless they
+        // are more than 2^24 apart, and then by less than 2^-52 of the sum
+        double dx[4] = {0.0, 0.0, 0.0, 0.0}, dy[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             const float2 a = lds_bin(bins_warp + lane * kSlotBytes + ((i + lane) & 31) * 8);
-            two_sum(hx[i & 3], lx[i & 3], a.x);
-            two_sum(hy[i & 3], ly[i & 3], a.y);
+            dx[i & 3] += (double)a.x;
+            dy[i & 3] += (double)a.y;
         }
-        wsum[warp * kPartStride + lane] = (((double)hx[0] + (double)lx[0]) + ((double)hx[1] + (double)lx[1])) +
-                                          (((double)hx[2] + (double)lx[2]) + ((double)hx[3] + (double)lx[3]));
-        wsum[warp * kPartStride + kCells + lane] = (((double)hy[0] + (double)ly[0]) + ((double)hy[1] + (double)ly[1])) +
-                                                   (((double)hy[2] + (double)ly[2]) + ((double)hy[3] + (double)ly[3]));
+        wsum[warp * kPartStride + lane] = (dx[0] + dx[1]) + (dx[2] + dx[3]);
+        wsum[warp * kPartStride + kCells + lane] = (dy[0] + dy[1]) + (dy[2] + dy[3]);
         // the warp's bins start the next pass at zero (done here, ahead of the wait for the totals)
         __syncwarp();
 #pragma unroll 8

@@ -567,6 +567,24 @@ def test_quantize_layers_rejects_a_bad_output_before_enqueuing_anything():
     assert binding.launch_count() == before
 
 
+def test_fit_refuses_a_layer_of_two_to_the_32_elements():
+    """The fit kernels index a layer with 32 bits: N * ldw = 2^32 is refused on the host, before the
+    workspace is looked at and before anything is enqueued (the buffers here are never touched)."""
+    small = torch.zeros(4096, dtype=torch.bfloat16, device=DEV)
+    d = dict(W=small.as_strided((1, 4096), (4096, 1)), I=torch.ones(4096, device=DEV), T01=torch.zeros(2, 16, device=DEV),
+             scales=torch.empty(256, dtype=torch.uint8, device=DEV), tensor_scale=torch.ones(1, device=DEV),
+             ws=torch.empty(1 << 20, dtype=torch.uint8, device=DEV))
+    arr = binding._layer_descs([d])
+    arr[0].N = 1 << 20                                   # 2^20 rows of 4096: exactly 2^32 elements
+    before = binding.launch_count()
+    rc = binding.lib().aaac_fit_layers(arr, 1, NVFP4, 16, 16, 2, 1, binding.INIT_GRID, None, None)
+    assert rc == 9, rc
+    arr[0].N = (1 << 20) - 1                             # one row less: now it is the workspace that is too small
+    rc = binding.lib().aaac_fit_layers(arr, 1, NVFP4, 16, 16, 2, 1, binding.INIT_GRID, None, None)
+    assert rc == 5, rc
+    assert binding.launch_count() == before
+
+
 def test_fit_layers_rejects_a_bad_layer_before_enqueuing_anything():
     W, X = layer(NVFP4, 16, 256, name="batchbad")
     good = dict(W=dev_bf16(W), I=torch.ones(256, device=DEV), T01=torch.zeros(2, 16, device=DEV),
