@@ -332,7 +332,23 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
     uint4 v[R];
     uint32_t sc[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
     uint32_t sgw[R];          // inner iteration: the row's stored selection bits
+    // Two forms of the row load, chosen per instantiation by measurement (the compiler schedules them
+    // differently): guarded, and unguarded with clamped indices -- a lane past the last column or row then
+    // reads the layer's last valid columns / row instead; columns past K carry I = 0, so their terms
+    // vanish, and rows past N are never processed.  INT4: clamped (8B-shaped stack 0.2155 -> 0.2113 s);
+    // NVFP4: guarded (clamped: 834 -> 802 Gweights/s on the benchmark layers).
+    constexpr bool kClampedLoads = MODE == AAAC_INT4;
     auto load_row = [&](int u, int slab, int rb) {
+        if constexpr (kClampedLoads) {
+            const int col0 = min(slab * 256 + lane * 8, K - 8);
+            const int row = min(rb * kRowsPerItem + warp * R + u, N - 1);
+            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + ((unsigned)row * (unsigned)p.ldw + (unsigned)col0)));
+            const unsigned gi = (unsigned)row * (unsigned)Gr + (unsigned)col0 / G;
+            if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];
+            else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
+            if (INNER) sgw[u] = __ldcg(p.sigw + (size_t)row * (size_t)slabs + slab);
+            return;
+        }
         const int col0 = slab * 256 + lane * 8;
         const int row = rb * kRowsPerItem + warp * R + u;
         v[u] = make_uint4(0, 0, 0, 0);
