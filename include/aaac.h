@@ -152,7 +152,8 @@ int aaac_fit_layer(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, i
 /*
  * Algorithm 1 lines 17-20: round the tables to BF16 (RNE of the FP32 values), recompute
  * sigma for every group with Eq. 8, store the nearest-entry index under the chosen table
- * (Eq. 6) as a 4-bit code, and put sigma into the sign bit of the scale.
+ * (Eq. 6) as a 4-bit code, and put sigma into the sign bit of the scale.  As for the fit, a layer
+ * must span fewer than 2^32 elements (N * ldw < 2^32), else AAAC_ERR_TOO_LARGE.
  *
  *   T01_f32   in   [2][16]
  *   T01_bf16  out  [2][16] BF16 bit patterns (64 bytes)

@@ -367,6 +367,8 @@ int aaac_pack_sel(const void* W, int64_t N, int64_t K, int64_t ldw, int mode, in
     if (!I || !T01_f32 || !T01_bf16 || !scales || !codes) return AAAC_ERR_NULL;
     if (mode == AAAC_NVFP4 && !tensor_scale) return AAAC_ERR_NULL;
     if (!aligned(I, 16) || !aligned(codes, 16) || !aligned(T01_bf16, 2)) return AAAC_ERR_ALIGN;
+    // the pack kernel, like the fit kernels, indexes a layer's elements with 32 bits
+    if ((unsigned long long)N * (unsigned long long)ldw >= (1ull << 32)) return AAAC_ERR_TOO_LARGE;
     rc = check_ws(ws, ws_bytes, carve(nullptr, mode, N, K).bytes);
     if (rc) return rc;
     return enqueue_pack(W, N, K, ldw, mode, sel_group, I, T01_f32, T01_bf16, scales, tensor_scale, codes, sigma_bits,

@@ -18,10 +18,11 @@
 // half-way between two different entries of their table, and of groups re-evaluated in double.
 //
 // Thread mapping.  The pass keeps no bins, so its lookup tables (512 bins) leave room for two
-// blocks of 12 warps per SM, and memory and table latency are hidden by the number of warps rather
+// blocks of 8 warps per SM, and memory and table latency are hidden by the number of warps rather
 // than by a hand-built pipeline: a warp walks down the rows of one 256-column slab (so its eight
-// importances stay in registers), one row at a time, the next row's load in flight; a lane takes 8
-// adjacent columns (one 128-bit load per row, one 32-bit store of 8 codes); the two errors travel
+// importances stay in registers), two rows per trip in registers of their own -- while one is worked
+// on, the other's load is in flight and nothing is copied -- with 32-bit element offsets advanced by
+// the row stride and no branch around the loads; a lane takes 8 adjacent columns (one 128-bit load per row, one 32-bit store of 8 codes); the two errors travel
 // as one packed FP32 pair.
 // Error sums go through one partial per block, added in block order by the last block to finish.
 #include "lookup.cuh"
@@ -30,7 +31,7 @@ namespace aaac {
 
 namespace {
 
-// warps per block (both instances run without register spills at 12; 16 is no faster)
+// warps per block
 #ifndef AAAC_PACK_WARPS
 #define AAAC_PACK_WARPS 8
 #endif
@@ -193,32 +194,30 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
             for (int o = LPG / 2; o; o >>= 1) isum += __shfl_xor_sync(0xFFFFFFFFu, isum, o);
             isum = __fmul_ru(isum * 1.0001f, g2);
         }
-        auto load = [&](int row, uint4& v, uint32_t& sc) {
-            v = make_uint4(0, 0, 0, 0);
-            sc = 0u;
-            if (col_ok && row < N) {
-                v = __ldcs(reinterpret_cast<const uint4*>(p.W + (size_t)row * (size_t)p.ldw + col0));
-                const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
-                if (MODE == AAAC_NVFP4) sc = reinterpret_cast<const uint8_t*>(p.scales)[gi];
-                else sc = reinterpret_cast<const uint16_t*>(p.scales)[gi];
-            }
+        // Element offsets of this lane's piece of the current row, advanced by the row stride (a layer of
+        // 2^32 elements or more is refused by the entry point); lanes past K read the slab's last valid
+        // columns instead (their importances are zero and they write nothing).
+        const unsigned col_ld = (unsigned)min(col0, K - 8);
+        const unsigned step_w = (unsigned)per_slab * (unsigned)p.ldw, step_g = (unsigned)per_slab * (unsigned)Gr;
+        const unsigned step_c = (unsigned)per_slab * (unsigned)(K >> 1);
+        const uint16_t* const Wp = p.W;
+        auto load = [&](unsigned wo, unsigned go, uint4& v, uint32_t& sc) {
+            v = __ldcs(reinterpret_cast<const uint4*>(Wp + wo));
+            if (MODE == AAAC_NVFP4) sc = reinterpret_cast<const uint8_t*>(p.scales)[go];
+            else sc = reinterpret_cast<const uint16_t*>(p.scales)[go];
         };
-        uint4 vn;
-        uint32_t scn;
-        load(my, vn, scn);
-        float ef = 0.f, eof = 0.f;            // the two error sums of up to 16 rows (double arithmetic is slow: one conversion per 16 rows)
+        float ef = 0.f, eof = 0.f;            // the two error sums of up to 16 rows (one conversion to double per 16 rows)
         int nrow = 0;
-        for (int row = my; row < N; row += per_slab) {
-            const uint4 v = vn;
-            const uint32_t sbits = MODE == AAAC_NVFP4 ? (scn & 0x7Fu) : (scn & 0x7FFFu);
-            load(row + per_slab, vn, scn);                 // the next row of this warp, in flight during this one
+        // one row: v and scv were loaded before; (wo, go) are the row's offsets, co the byte offset of its codes
+        auto do_row = [&](const uint4& v, uint32_t scv, int row, unsigned go, unsigned co) {
+            const uint32_t sbits = MODE == AAAC_NVFP4 ? (scv & 0x7Fu) : (scv & 0x7FFFu);
             float sval, rinv;
             if (MODE == AAAC_NVFP4) {
                 sval = slut[sbits];
                 rinv = S.rlut[sbits];
             } else {
                 sval = __uint_as_float(sbits << 16);
-                rinv = sbits ? __frcp_rn(sval) : 0.f;       // lanes past K hold no scale
+                rinv = __frcp_rn(sval);
             }
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
             float x[8];
@@ -272,13 +271,12 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
                 if (col_ok && (lane & 15) == 0)
                     p.sigma_bits[(size_t)row * (size_t)(K >> 7) + (uint32_t)col0 / 128u] = (uint8_t)(bb >> (lane >> 1));
             }
-            if (!col_ok) continue;
+            if (!col_ok) return;
             if ((lane % LPG) == 0) {
                 // both error sums from the group's smaller error: sum I (w - w^)^2 = s^2 sum I (w~ - T)^2
                 ef += emin;
                 eof = __fmaf_rn(emin, __fmul_rn(sval, sval), eof);
             }
-            if (++nrow == 16) { Eacc += (double)ef; Eout += (double)eof; ef = 0.f; eof = 0.f; nrow = 0; }
             // codes (Eq. 6): the entry index rides in the low mantissa bits of the chosen constant
             uint32_t word = 0;
 #pragma unroll
@@ -287,13 +285,35 @@ __global__ void __launch_bounds__(NW * 32, kPackBlocksPerSM) pack_kernel(const P
                 unpack2(pq[j], cP, cQ);
                 word |= (__float_as_uint(sg ? cQ : cP) & kIdxMask) << (4 * j);
             }
-            *reinterpret_cast<uint32_t*>(p.codes + (((size_t)row * (size_t)K + col0) >> 1)) = word;
+            *reinterpret_cast<uint32_t*>(p.codes + co) = word;
             if (SEL == G && (lane % LPG) == 0) {
-                const size_t gi = (size_t)row * (size_t)Gr + (uint32_t)col0 / G;
                 if (MODE == AAAC_NVFP4)
-                    reinterpret_cast<uint8_t*>(p.scales)[gi] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
+                    reinterpret_cast<uint8_t*>(p.scales)[go] = (uint8_t)(sbits | (sg ? 0x80u : 0u));
                 else
-                    reinterpret_cast<uint16_t*>(p.scales)[gi] = (uint16_t)(sbits | (sg ? 0x8000u : 0u));
+                    reinterpret_cast<uint16_t*>(p.scales)[go] = (uint16_t)(sbits | (sg ? 0x8000u : 0u));
+            }
+        };
+        // Two rows per trip, each in registers of its own: while one is worked on the other's load is in
+        // flight, and nothing is copied.  Past the warp's last row the same row is fetched again (unused).
+        if (my < N) {
+            unsigned wo = (unsigned)my * (unsigned)p.ldw + col_ld, go = (unsigned)my * (unsigned)Gr + col_ld / G;
+            unsigned co = ((unsigned)my * (unsigned)K + (unsigned)col0) >> 1;
+            uint4 va, vb;
+            uint32_t sa, sb;
+            load(wo, go, va, sa);
+            for (int row = my; row < N; row += 2 * per_slab) {
+                const bool more1 = row + per_slab < N;
+                const unsigned wo1 = more1 ? wo + step_w : wo, go1 = more1 ? go + step_g : go;
+                load(wo1, go1, vb, sb);
+                do_row(va, sa, row, go, co);
+                if (!more1) break;
+                const bool more2 = row + 2 * per_slab < N;
+                const unsigned wo2 = more2 ? wo1 + step_w : wo1, go2 = more2 ? go1 + step_g : go1;
+                load(wo2, go2, va, sa);
+                do_row(vb, sb, row + per_slab, go1, co + step_c);
+                wo = wo2; go = go2; co += 2 * step_c;
+                nrow += 2;
+                if (nrow >= 16) { Eacc += (double)ef; Eout += (double)eof; ef = 0.f; eof = 0.f; nrow = 0; }
             }
         }
         Eacc += (double)ef;

@@ -582,6 +582,14 @@ def test_fit_refuses_a_layer_of_two_to_the_32_elements():
     arr[0].N = (1 << 20) - 1                             # one row less: now it is the workspace that is too small
     rc = binding.lib().aaac_fit_layers(arr, 1, NVFP4, 16, 16, 2, 1, binding.INIT_GRID, None, None)
     assert rc == 5, rc
+    # the pack pass has the same limit
+    codes = torch.empty(4096, dtype=torch.uint8, device=DEV)
+    Tb = torch.empty(2, 16, dtype=torch.uint16, device=DEV)
+    args = lambda N: (d["W"].data_ptr(), N, 4096, 4096, NVFP4, 16, d["I"].data_ptr(), d["T01"].data_ptr(), Tb.data_ptr(),
+                      d["scales"].data_ptr(), d["tensor_scale"].data_ptr(), codes.data_ptr(), None, None, d["ws"].data_ptr(),
+                      d["ws"].numel(), None)
+    assert binding.lib().aaac_pack(*args(1 << 20)) == 9
+    assert binding.lib().aaac_pack(*args((1 << 20) - 1)) == 5
     assert binding.launch_count() == before
 
 
