@@ -9,9 +9,11 @@
  * Conventions for every entry point
  *   - Pointers are DEVICE pointers unless the name ends in _host.  The caller owns every
  *     buffer; the library allocates no device memory and keeps no per-call state, except for
- *     three process-wide diagnostics / conveniences that are documented where they are declared:
+ *     four process-wide diagnostics / conveniences that are documented where they are declared:
  *     the event table of aaac_timing_begin / aaac_timing_end, the launch counter of
- *     aaac_launch_count, and the built-in scratch array of aaac_act_stats_noalloc.
+ *     aaac_launch_count, the built-in scratch array of aaac_act_stats_noalloc, and the seven
+ *     streams and eight events per device that aaac_fit_layers / aaac_quantize_layers create at
+ *     their first call with more than one layer.
  *   - W is [N x K] row-major BF16 (N = output rows, K = input channels, y = x W^T, Sec. 3.1),
  *     leading dimension ldw (elements).  Groups are g contiguous elements of a row.
  *     X is [T x K] row-major BF16 calibration activations, leading dimension ldx.
