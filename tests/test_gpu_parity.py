@@ -492,6 +492,15 @@ def test_fit_layers_more_layers_than_one_launch_takes_and_inner_refinement():
         assert np.allclose(host(d["err_trace"])[:2], o["trace"], rtol=1e-4)
 
 
+def carved_importance(d):
+    """The importances of a layer as aaac_act_stats gives them for the X the batch call was given
+    (the batch call keeps its own copy inside the layer's workspace)."""
+    I = torch.empty(d["X"].shape[1], dtype=torch.float32, device=DEV)
+    binding.act_stats(d["X"], I, binding.alloc_workspace(NVFP4, 8, d["X"].shape[1], d["X"].shape[0]))
+    torch.cuda.synchronize()
+    return I
+
+
 def run_quantize_batch(cases, mode, rounds, init, sel_group=None, what_pad=0):
     """aaac_quantize_layers on a list of (W, X) cases, importances from X inside the call."""
     g = 128 if mode == INT4 else 16
@@ -606,27 +615,28 @@ def test_fit_layers_rejects_a_bad_layer_before_enqueuing_anything():
 
 
 def test_config2_layers_in_one_batch_full_size():
-    """The benchmark's three layers fitted in one call (the launch configuration the benchmark times):
-    each against the whole-layer oracle."""
+    """The benchmark's step as the benchmark makes it -- its three layers through aaac_quantize_layers in one
+    call, importances from X, scales, quantile start, the 20 rounds of all three in one launch, pack and
+    reconstruction -- with every output of every layer against the whole-layer oracle."""
+    names = ("q_proj", "gate_proj", "down_proj")
     cases, oracles = [], []
-    for which in ("q_proj", "gate_proj", "down_proj"):
+    for which in names:
         c = synth.config2_layer(which)
-        o = oracle.fit_layer(c["W"], NVFP4, 16, c["rounds"], X=c["X"], init="quantile")
-        cases.append((c["W"], o["I"]))
-        oracles.append(o)
-    for which, d, o in zip(("q_proj", "gate_proj", "down_proj"), run_fit_batch(cases, NVFP4, 20, binding.INIT_QUANTILE), oracles):
+        oracles.append(oracle.fit_layer(c["W"], NVFP4, 16, c["rounds"], X=c["X"], init="quantile"))
+        cases.append((c["W"], c["X"]))
+    for which, d, o in zip(names, run_quantize_batch(cases, NVFP4, 20, binding.INIT_QUANTILE), oracles):
+        assert np.allclose(host(carved_importance(d)), o["I"], rtol=1e-6, atol=0), f"{which}: importances differ"
         ok, worst = table_close(host(d["T01"]), o["T"])
         assert ok, f"{which}: tables differ: worst {worst:.3e}"
         tr = host(d["err_trace"])[:20]
         assert np.allclose(tr, o["trace"], rtol=1e-4, atol=0) and np.all(tr[1:] <= tr[:-1] * (1 + 1e-6))
-        Tb = torch.empty(2, 16, dtype=torch.uint16, device=DEV)
-        codes = torch.empty(d["W"].shape[0], d["W"].shape[1] // 2, dtype=torch.uint8, device=DEV)
-        binding.pack(d["W"], NVFP4, I=d["I"], T01=d["T01"], T01_bf16=Tb, scales=d["scales"], tensor_scale=d["tensor_scale"],
-                     codes=codes, ws=d["ws"])
-        differ = int(np.sum(host(Tb) != o["T_bf16"]))
+        differ = int(np.sum(host(d["T01_bf16"]) != o["T_bf16"]))
         print(f"batched {which}: worst table deviation {worst:.2e}, BF16 entries that differ {differ}")
         assert differ == 0
-        assert np.array_equal(host(codes), o["codes"]) and np.array_equal(host(d["scales"]), o["scales"])
+        assert np.array_equal(host(d["codes"]), o["codes"]) and np.array_equal(host(d["scales"]), o["scales"])
+        assert np.isclose(host(d["err_out"])[0], o["E_final"], rtol=1e-4)
+        want = oracle.dequant(o["codes"], o["scales"], o["tensor_scale"], o["T_bf16"], NVFP4, 16)
+        assert np.array_equal(host(d["What"].contiguous()), want), f"{which}: reconstruction differs"
 
 
 # ------------------------------------------------------------------ inner refinement (n_inner > 1)
