@@ -96,6 +96,7 @@ struct FitParams {
     int tail_item0, tail_quarters;   // items from tail_item0 on are dealt out a quarter (one row per warp) per block
 };
 
+constexpr uint32_t kLut1At = 65536;                    // shared address of the bin table (see fit_rounds_body)
 constexpr int kMaxFitBlocks = 1024;                   // grid limit: block sums are added as 32-bit limbs, the arrivals counted in 16 bits
 constexpr int kLimbs = 3;                             // a sum is a 96-bit two's-complement fixed-point number
 constexpr unsigned kDefaultSpinLimit = 1u << 23;      // polls of >= 32 ns each: several seconds
@@ -247,16 +248,34 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
     __shared__ FitTables S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // 32-bit shared addresses.  Slot offsets carry the address of this lane's column of the
-    // {P, Q} table, so a lookup there needs no further arithmetic.
+    // 32-bit shared addresses.  The bin table sits at a shared address that is a multiple of its own
+    // span (64 KB), so that a lookup's address -- bin bits, the lane's copy and the table base -- is one
+    // three-input logic instruction; the bins of the first warps fill the space below it, the other
+    // warps' bins, the {P, Q} table and the near-tie lists follow it.  Slot offsets carry the address of
+    // this lane's column of the {P, Q} table, so a lookup there needs no further arithmetic.
+    static_assert(kLut1Bytes == (int)kLut1At, "the bin table spans exactly the alignment of its address");
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(dyn);
-    const uint32_t lut1_copy = (lane & (REP - 1)) * 8;                                 // this lane's copy of a bin's entry; | bin * REP * 8
-    const uint32_t lut2_addr = sm_base + kLut1Bytes;                                   // the {P, Q} table
-    const uint32_t bins_warp = sm_base + kLut1Bytes + kLut2Bytes + warp * kBinBytes;
+    uint32_t dyn_size;
+    asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_size));
+    const uint32_t gap = kLut1At - sm_base;                                            // bytes of the dynamic region below the table
+    const int n_low = min(NW, (int)(gap / (uint32_t)kBinBytes));                       // warps whose bins lie below the table
+    const uint32_t hi_base = kLut1At + kLut1Bytes;
+    const uint32_t lut2_addr = hi_base + (uint32_t)(NW - n_low) * kBinBytes;           // the {P, Q} table
+    const uint32_t lists_at = lut2_addr + kLut2Bytes;
+    if (sm_base > kLut1At || lists_at + NW * (kDeferCap * 8) > sm_base + dyn_size) {
+        // the layout does not fit the shared memory this launch was given (the same for every block, so
+        // all of them leave before any of them waits): reported like a wait that ran out -- no valid result
+        if (bid == 0 && threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, AAAC_DEV_TIMEOUT);
+        return;
+    }
+    unsigned char* const lut1_mem = dyn + gap;
+    unsigned char* const lut2_mem = dyn + (lut2_addr - sm_base);
+    const uint32_t lut1_or = kLut1At | ((lane & (REP - 1)) * 8);                        // table base | this lane's copy of a bin's entry; | bin * REP * 8
+    const uint32_t bins_warp = warp < n_low ? sm_base + warp * kBinBytes : hi_base + (uint32_t)(warp - n_low) * kBinBytes;
     const uint32_t bins_lane = bins_warp + lane * 8;                                   // + cell * 256
     const uint32_t spare_lane = bins_lane + kSpareSlot * kSlotBytes;                   // sink of the near-tie groups' rows
-    const uint32_t list_addr = sm_base + kLut1Bytes + kLut2Bytes + NW * kBinBytes + warp * (kDeferCap * 8);
-    double* wsum = reinterpret_cast<double*>(dyn);         // [NW][kPartStride], over the first table
+    const uint32_t list_addr = lists_at + warp * (kDeferCap * 8);
+    double* wsum = reinterpret_cast<double*>(lut1_mem);    // [NW][kPartStride], over the first table
 
     // 32-bit index arithmetic throughout (N, K < 2^31); only the final element offsets are 64-bit
     const int N = (int)p.N, K = (int)p.K;
@@ -288,7 +307,7 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
         for (int k = tid; k < K; k += NT) mx = fmaxf(mx, fabsf(__ldg(p.I + k)));
 #pragma unroll
         for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        float* red = reinterpret_cast<float*>(dyn);
+        float* red = reinterpret_cast<float*>(lut1_mem);
         if (lane == 0) red[warp] = mx;
         __syncthreads();
         if (tid == 0) {
@@ -317,7 +336,7 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
         p.acc[(size_t)((pass_no + 1u) % 3u) * kAccBuffer + (size_t)(tid - 256) * kAccStride] = 0ull;
         __threadfence();
     }
-    build_tables<MODE, NW, REP, NB>(S, dyn);
+    build_tables<MODE, NW, REP, NB>(S, lut1_mem, lut2_mem);
     // near-tie bound: sqrt(a b) <= (kappa a + b / kappa) / 2, so the bound of the header comment is at
     // most g1 * (E0 + E1) + g2 * sum I, with kappa = 1/8 (about the usual |w~ - entry|)
     const float g1 = 0x1p-24f * __fmaf_ru(S.tmax283, 4.f, 16.f), g2 = 0x1p-24f * __fmul_ru(S.tmax283, 0.0625f);
@@ -332,23 +351,9 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
     uint4 v[R];
     uint32_t sc[R];           // NVFP4: scale byte; INT4: bits of the reciprocal scale
     uint32_t sgw[R];          // inner iteration: the row's stored selection bits
-    // Two forms of the row load, chosen per instantiation by measurement (the compiler schedules them
-    // differently): guarded, and unguarded with clamped indices -- a lane past the last column or row then
-    // reads the layer's last valid columns / row instead; columns past K carry I = 0, so their terms
-    // vanish, and rows past N are never processed.  INT4: clamped (8B-shaped stack 0.2155 -> 0.2113 s);
-    // NVFP4: guarded (clamped: 834 -> 802 Gweights/s on the benchmark layers).
-    constexpr bool kClampedLoads = MODE == AAAC_INT4;
+    // (An unguarded form with clamped indices was measured too: faster for some instantiations, slower
+    // for others, depending on what else the kernel held; the guarded form is the one kept.)
     auto load_row = [&](int u, int slab, int rb) {
-        if constexpr (kClampedLoads) {
-            const int col0 = min(slab * 256 + lane * 8, K - 8);
-            const int row = min(rb * kRowsPerItem + warp * R + u, N - 1);
-            v[u] = __ldcs(reinterpret_cast<const uint4*>(p.W + ((unsigned)row * (unsigned)p.ldw + (unsigned)col0)));
-            const unsigned gi = (unsigned)row * (unsigned)Gr + (unsigned)col0 / G;
-            if (MODE == AAAC_NVFP4) sc[u] = p.scales[gi];
-            else sc[u] = __float_as_uint(__ldg(p.rinv + gi));
-            if (INNER) sgw[u] = __ldcg(p.sigw + (size_t)row * (size_t)slabs + slab);
-            return;
-        }
         const int col0 = slab * 256 + lane * 8;
         const int row = rb * kRowsPerItem + warp * R + u;
         v[u] = make_uint4(0, 0, 0, 0);
@@ -440,8 +445,7 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
                 x[j] = __fmul_rn((j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]), rinv);
                 // (bin bits | lane's copy) is one three-input logic instruction, and the table's base, the
                 // same for every lane, can ride in the load's address: no add per weight
-                const uint32_t off = ((uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask) | lut1_copy;
-                e1v[j] = lds_table_u2(sm_base + off);
+                e1v[j] = lds_table_u2(((uint32_t)__float_as_int(__fmaf_rn(x[j], kBinsPerUnit, kMagic)) & kBinMask) | lut1_or);
             }
         };
         // same, then refill the row's registers from the next item
@@ -742,11 +746,27 @@ __global__ void export_tables_kernel(const Ctrl* ctrl, float* T01) {
     if (threadIdx.x < 2 * kM) T01[threadIdx.x] = (float)ctrl->T[threadIdx.x];
 }
 
+// The fit kernels place their tables at fixed shared addresses and take all the shared memory a block
+// may have beyond their static part (one block per SM either way); the kernel checks that its layout fits.
+cudaError_t fit_dynamic_smem(const void* kern, size_t* bytes) {
+    cudaFuncAttributes a;
+    cudaError_t e = cudaFuncGetAttributes(&a, kern);
+    if (e != cudaSuccess) return e;
+    int dev = 0, optin = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+    if ((size_t)optin <= a.sharedSizeBytes) return cudaErrorInvalidValue;
+    *bytes = (size_t)optin - a.sharedSizeBytes;
+    return cudaSuccess;
+}
+
 template <int MODE, int SEL, int NW, int REP, int KIND>
 cudaError_t launch_variant(FitParams& p, unsigned grid, cudaStream_t st) {
-    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kLut2Bytes + (size_t)NW * kBinSlots * kSlotBytes + (size_t)NW * kDeferCap * 8;
     auto kern = fit_rounds_kernel<MODE, SEL, NW, REP, KIND>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    size_t smem = 0;
+    cudaError_t e = fit_dynamic_smem(reinterpret_cast<const void*>(kern), &smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&p};
     note_launch();
@@ -838,9 +858,11 @@ cudaError_t launch_fit_rounds(const uint16_t* W, int64_t N, int64_t K, int64_t l
 template <int MODE, int SEL>
 static cudaError_t launch_batch_variant(FitBatch& b, unsigned grid, cudaStream_t st) {
     constexpr int NW = AAAC_FIT_WARPS, REP = AAAC_FIT_REP;
-    constexpr size_t smem = (size_t)REP * AAAC_FIT_BINS * 8 + kLut2Bytes + (size_t)NW * kBinSlots * kSlotBytes + (size_t)NW * kDeferCap * 8;
     auto kern = fit_batch_kernel<MODE, SEL, NW, REP>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    size_t smem = 0;
+    cudaError_t e = fit_dynamic_smem(reinterpret_cast<const void*>(kern), &smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     void* args[] = {&b};
     note_launch();

@@ -124,7 +124,7 @@ struct FitTables {
 
 // Builds every lookup table of the round from the current tables in S.Td.
 template <int MODE, int NW, int REP, int NB = kNBins>
-__device__ void build_tables(FitTables& S, unsigned char* dyn) {
+__device__ void build_tables(FitTables& S, unsigned char* lut1_mem, unsigned char* lut2_mem) {
     constexpr int NT = NW * 32;
     const int tid = threadIdx.x;
     if (tid < kNBP) {
@@ -162,7 +162,7 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
         S.exact[rank] = S.tmp_exact[tid];
     }
     __syncthreads();
-    float2* lut2 = reinterpret_cast<float2*>(dyn + (size_t)REP * NB * 8);
+    float2* lut2 = reinterpret_cast<float2*>(lut2_mem);
     if (tid < kJSlots) {
         float P = __int_as_float(0x7FC00000), Q = P;
         if (tid < kNJ) {
@@ -191,8 +191,8 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
     // of bank conflicts (one thread writing the REP copies of its bin would serialise 32-fold).
     static_assert(NB * 8 <= kLut2Bytes, "the per-bin entries are staged in the {P, Q} table's space");
     static_assert(REP == kPqCols, "copy c of a bin's entry carries the address of column c of the {P, Q} table");
-    uint2* binval = reinterpret_cast<uint2*>(dyn + (size_t)REP * NB * 8);
-    const uint32_t lut2_addr = (uint32_t)__cvta_generic_to_shared(dyn + (size_t)REP * NB * 8);
+    uint2* binval = reinterpret_cast<uint2*>(lut2_mem);
+    const uint32_t lut2_addr = (uint32_t)__cvta_generic_to_shared(lut2_mem);
     constexpr float h = 0.5f / (float)(REP * 8);
     constexpr float kHalf = (float)(NB / 2), kWidth = 16.f / (float)NB;
     for (int b = tid; b < NB; b += NT) {
@@ -214,7 +214,7 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
     }
     __syncthreads();
     {
-        uint4* lut1v = reinterpret_cast<uint4*>(dyn);    // two copies (columns 2 i mod REP and the next) per store
+        uint4* lut1v = reinterpret_cast<uint4*>(lut1_mem);    // two copies (columns 2 i mod REP and the next) per store
         for (int i = tid; i < NB * REP / 2; i += NT) {
             const uint2 e = binval[(2 * i) / REP];
             const uint32_t col = (uint32_t)((2 * i) % REP) * 8u;
@@ -229,6 +229,12 @@ __device__ void build_tables(FitTables& S, unsigned char* dyn) {
         lut2[i] = S.pq32[J];
     }
     __syncthreads();
+}
+
+// the two tables one after the other in one buffer
+template <int MODE, int NW, int REP, int NB = kNBins>
+__device__ __forceinline__ void build_tables(FitTables& S, unsigned char* dyn) {
+    build_tables<MODE, NW, REP, NB>(S, dyn, dyn + (size_t)REP * NB * 8);
 }
 
 // address of column (lane mod 16) of interval J's entry in the {P, Q} table that starts at lut2_addr
