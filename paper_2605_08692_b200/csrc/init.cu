@@ -108,7 +108,10 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     __shared__ unsigned long long base[kQReq];
     __shared__ uint32_t nbuf;
     __shared__ uint32_t okmin[kQReq], okmax[kQReq];       // smallest / largest key of the slots without list space
+    __shared__ float rl[128];                             // NVFP4: reciprocal of the effective scale per E4M3 code
     const int tid = threadIdx.x, lane = tid & 31;
+    const float s_t = ctrl->s_t;
+    if (MODE == AAAC_NVFP4 && tid < 128) rl[tid] = __frcp_rn(__fmul_rn(e4m3_value((uint32_t)tid), s_t));
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(slot_of_bin);
         for (int i = tid; i < kQBins / 4; i += blockDim.x) sm[i] = src[i];
@@ -117,7 +120,6 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     }
     __syncthreads();
     const uint8_t* sm_slot = reinterpret_cast<const uint8_t*>(sm);
-    const float s_t = ctrl->s_t;
     const int64_t slabs = (K + 255) / 256, items = N * slabs, Gr = K / G;
     const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + tid) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -139,14 +141,17 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     };
 
     SlabWalk it(warp0, nwarps, slabs);
-    auto fetch = [&](uint4& vv, float& rr, bool& okk) {
+    // (the scale travels as its stored bits: nothing waits for the load before the row is worked on)
+    auto fetch = [&](uint4& vv, uint32_t& ss, bool& okk) {
         const int64_t row = it.row, col = (int64_t)it.slab * 256 + lane * 8;
         okk = row < N && col < K;
         vv = make_uint4(0, 0, 0, 0);
-        rr = 0.f;
+        ss = 0u;
         if (okk) {
             vv = __ldg(reinterpret_cast<const uint4*>(W + row * ldw + col));
-            rr = group_rinv<MODE>(scales, row * Gr + col / G, s_t);
+            const int64_t gi = row * Gr + col / G;
+            if (MODE == AAAC_INT4) ss = reinterpret_cast<const uint16_t*>(scales)[gi];
+            else ss = reinterpret_cast<const uint8_t*>(scales)[gi];
         }
         it.next();
     };
@@ -154,7 +159,9 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     // for, so the AND of the eight bytes tells whether the lane holds a candidate; a lane that does
     // walks only its candidates (one, nearly always), found by a bit scan of the packed bytes, and
     // recomputes w~ of that weight alone.
-    auto take = [&](const uint4& v, float r) {
+    auto take = [&](const uint4& v, uint32_t ss) {
+        // the reciprocal group_rinv would give for these scale bits
+        const float r = MODE == AAAC_INT4 ? __frcp_rn(__uint_as_float((ss & 0x7FFFu) << 16)) : rl[ss & 0x7Fu];
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
         uint32_t sl[8], all = 0x80u;
 #pragma unroll
@@ -197,13 +204,13 @@ quantile_collect_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, in
     // is processed.  The warps of a block meet only every kStageEvery iterations, to empty the
     // stage once it is half full (the vote makes the decision the same for every thread).
     uint4 va, vb;
-    float ra, rb;
+    uint32_t ra, rb;
     bool oka, okb;
     fetch(va, ra, oka);
     fetch(vb, rb, okb);
     for (int64_t k = 0; k < iters; ++k) {
         uint4 vna, vnb;
-        float rna, rnb;
+        uint32_t rna, rnb;
         bool okna, oknb;
         fetch(vna, rna, okna);
         fetch(vnb, rnb, oknb);
