@@ -162,6 +162,8 @@ scales_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t
         ctrl->s_t = s_t;
         if (tensor_scale) tensor_scale[0] = s_t;
     }
+    __shared__ float rl[128];                          // NVFP4: fl32(1 / (E4M3 value * s_t)) per scale code, as the later passes form it
+    if (MODE == AAAC_NVFP4 && threadIdx.x < 128) rl[threadIdx.x] = __frcp_rn(__fmul_rn(e4m3_value(threadIdx.x), s_t));
     __syncthreads();
     bool bad = false;
     SlabWalk it(warp0, nwarps, slabs);
@@ -203,7 +205,7 @@ scales_hist_kernel(const uint16_t* __restrict__ W, int64_t N, int64_t K, int64_t
             const float x = __fdiv_rn(a, d6);
             uint32_t q = e4m3_encode(x);
             if (q <= 1u) q = (x > 1.25f * 0x1p-9f) ? 2u : 1u;
-            r = __frcp_rn(__fmul_rn(e4m3_value(q), s_t));
+            r = rl[q];
             if ((lane % LPG) == 0) reinterpret_cast<uint8_t*>(scales)[gi] = (uint8_t)q;
         }
         const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
