@@ -550,7 +550,8 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
         };
 
         if (nrows == R && whole) {
-            // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..3] L2(1) B(0)[4..7] M(1) | ... | B(R-1)
+            // full item: L1(0) L2(0) M(0) | L1(1) B(0)[0..1] L2(1) B(0)[2..7] M(1) | ... | B(R-1)
+            // (where the second lookups cut into the previous row's bin updates was chosen by measurement: 2 + 6)
             L1n(0);
             L2();
             M(row0, mt[0], ba[0]);
@@ -558,9 +559,9 @@ __device__ __forceinline__ void fit_rounds_body(const FitParams& p, const unsign
             for (int u = 1; u < R; ++u) {
                 const int prev = (u - 1) & 1, cur = u & 1;
                 L1n(u);
-                B(mt[prev], ba[prev], 0, 4);
+                B(mt[prev], ba[prev], 0, 2);
                 L2();
-                B(mt[prev], ba[prev], 4, 8);
+                B(mt[prev], ba[prev], 2, 8);
                 M(row0 + u, mt[cur], ba[cur]);
             }
             B(mt[(R - 1) & 1], ba[(R - 1) & 1], 0, 8);
