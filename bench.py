@@ -253,18 +253,15 @@ def run_stack(args, which, emit=True):
                       err=torch.zeros(2, dtype=torch.float64, device=dev),
                       bits=torch.empty(N, K // (8 * sel), dtype=torch.uint8, device=dev) if sel and sel != g else None,
                       ws=binding.alloc_workspace(mode, N, K, tokens, dev))
-    Iv = {k: torch.empty(x.shape[1], dtype=torch.float32, device=dev) for k, x in X.items()}
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    descs = [dict(W=Ws[n], I=Iv[xin], T01=out[n]["T01"], scales=out[n]["scales"], tensor_scale=out[n]["ts"], ws=out[n]["ws"],
+    # the seven linears of a decoder layer are independent: one aaac_quantize_layers call (importances -- once per
+    # distinct input: q, k, v share theirs, gate and up too --, scales, start, rounds in one launch, pack)
+    descs = [dict(W=Ws[n], X=X[xin], T01=out[n]["T01"], scales=out[n]["scales"], tensor_scale=out[n]["ts"], ws=out[n]["ws"],
                   T01_bf16=out[n]["Tb"], codes=out[n]["codes"], err_out=out[n]["err"], sigma_bits=out[n]["bits"])
              for n, N, K, xin in lin]
 
     def decoder_layer():
-        for k, x in X.items():
-            binding.act_stats(x, Iv[k], out["down" if k == "down" else "q"]["ws"], dev_status=status)
-        # the seven linears of a decoder layer are independent: one aaac_quantize_layers call (scales, start,
-        # rounds in one launch, pack)
         binding.quantize_layers(descs, mode, n_outer=rounds, n_inner=n_inner, init=binding.INIT_QUANTILE, dev_status=status,
                                 sel_group=sel)
 
@@ -297,7 +294,7 @@ def run_stack(args, which, emit=True):
                        "linears": 7 * L, "weights": wl * L, "rounds": rounds, "n_inner": n_inner},
             "gweights_per_s_per_round": wl * L * rounds * n_inner / wall / 1e9, "clocks": clocks,
             "gpu_launches": launches_per_layer * L}
-    del X, Ws, out, Iv
+    del X, Ws, out
     torch.cuda.empty_cache()
     if emit:
         print(json.dumps(line), flush=True)

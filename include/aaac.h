@@ -221,7 +221,9 @@ int aaac_dequant_sel(const uint8_t* codes, const void* scales, const uint8_t* si
  * share of the blocks, so that the cost of a round that does not depend on the layer's size is
  * paid once per batch and small layers do not leave most of the GPU idle; more layers, and
  * n_inner > 1, are run in turn.  Scales, importances (from X where I is NULL) and start tables
- * are computed per layer exactly as by aaac_fit_layer_sel.  With more than one layer these
+ * are computed per layer exactly as by aaac_fit_layer_sel, except that layers given the same
+ * activations (the same X, T, K and ldx, with I == NULL) share their importances, which are
+ * computed once (into the workspace of the first of them).  With more than one layer these
  * per-layer passes are queued on up to seven streams the library keeps per device (created at the
  * first such call), forked from `stream` and joined back to it before the fit launch: seen from
  * `stream`, the call is ordered like any other.

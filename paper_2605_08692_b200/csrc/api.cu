@@ -256,12 +256,26 @@ int check_fit_layer(const aaac_layer& L, int mode, int group, int sel_group, int
     return check_ws(L.ws, L.ws_bytes, carve(nullptr, mode, L.N, L.K).bytes);
 }
 
-// Alg. 1 lines 1-5 of one layer: importance (if from X), scales, start tables; returns the importance used
+// Layers of a batch that are given the same activations (pointer, T, K, ldx) share their importances:
+// they are computed once, into the workspace of the first such layer.  Returns that layer's index
+// (l itself for a layer with importances of its own or activations nobody before it has).
+int importance_owner(const aaac_layer* layers, int l) {
+    const aaac_layer& L = layers[l];
+    if (L.I) return l;
+    for (int k = 0; k < l; ++k) {
+        const aaac_layer& M = layers[k];
+        if (!M.I && M.X == L.X && M.T == L.T && M.K == L.K && M.ldx == L.ldx) return k;
+    }
+    return l;
+}
+
+// Alg. 1 lines 1-5 of one layer: importance (if from X and not shared with an earlier layer, whose
+// `shared_I` is then passed), scales, start tables; returns the importance used
 int prepare_fit_layer(const aaac_layer& L, int mode, int init, uint32_t* dev_status, const Workspace& w, cudaStream_t st,
-                      const float** I_used) {
+                      const float* shared_I, const float** I_used) {
     const uint16_t* Wp = static_cast<const uint16_t*>(L.W);
     if (cudaMemsetAsync(w.ctrl, 0, sizeof(Ctrl), st) != cudaSuccess) return AAAC_ERR_CUDA;
-    const float* I = L.I;
+    const float* I = L.I ? L.I : shared_I;
     if (!I) {
         if (launch_act_stats(static_cast<const uint16_t*>(L.X), L.T, L.K, L.ldx, w.I, 0, dev_status, w, st) != cudaSuccess)
             return AAAC_ERR_CUDA;
@@ -293,7 +307,11 @@ int aaac_fit_layers(const aaac_layer* layers, int n_layers, int mode, int group,
             const aaac_layer& L = layers[l];
             const Workspace w = carve(L.ws, mode, L.N, L.K, L.ws_bytes);
             const float* I = nullptr;
-            rc = prepare_fit_layer(L, mode, init, dev_status, w, lanes.of(l), &I);
+            // (the passes queued here do not read the importances; the fit launch, after the join, does)
+            const int owner = importance_owner(layers, l);
+            const float* shared_I = owner == l ? nullptr
+                                               : carve(layers[owner].ws, mode, layers[owner].N, layers[owner].K, layers[owner].ws_bytes).I;
+            rc = prepare_fit_layer(L, mode, init, dev_status, w, lanes.of(l), shared_I, &I);
             args[l] = FitLayerArgs{static_cast<const uint16_t*>(L.W), L.N, L.K, L.ldw, L.scales, I, L.err_trace, L.T01, w};
         }
         if (!lanes.join() && rc == AAAC_OK) rc = AAAC_ERR_CUDA;
@@ -398,8 +416,9 @@ int aaac_quantize_layers(const aaac_layer* layers, const aaac_layer_out* outs, i
     for (int l = 0; l < n_layers && rc == AAAC_OK; ++l) {
         const aaac_layer& L = layers[l];
         const aaac_layer_out& O = outs[l];
-        // the importance the fit used: the caller's, or the one the fit computed from X into the workspace
-        const float* I = L.I ? L.I : carve(L.ws, mode, L.N, L.K, L.ws_bytes).I;
+        // the importance the fit used: the caller's, or the one the fit computed from X into a workspace
+        const aaac_layer& Lo = layers[importance_owner(layers, l)];
+        const float* I = L.I ? L.I : carve(Lo.ws, mode, Lo.N, Lo.K, Lo.ws_bytes).I;
         uint8_t* sg = sel_group == group ? nullptr : O.sigma_bits;
         rc = enqueue_pack(L.W, L.N, L.K, L.ldw, mode, sel_group, I, L.T01, O.T01_bf16, L.scales, L.tensor_scale, O.codes, sg,
                           O.err_out, O.stats, L.ws, L.ws_bytes, lanes.of(l));

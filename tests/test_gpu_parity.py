@@ -563,6 +563,45 @@ def test_quantize_layers_whole_path_matches_oracle_per_layer(mode, sel):
         assert bool((d["What_full"][:, o["codes"].shape[1] * 2:] == 7.0).all()), f"{label}: wrote past a row of What"
 
 
+def test_quantize_layers_share_the_importances_of_a_common_input():
+    """Layers of a batch that read the same activations (q, k and v of a decoder layer): the importances
+    are computed once -- two kernels fewer per further layer -- and every layer still matches the oracle."""
+    K = 512
+    X = synth.activations(96, K, 11, "shared/X", kind="lognormal", massive_frac=0.005)
+    Ws = [synth.weights(N, K, 11, f"shared/W{i}", outlier_frac=0.01) for i, N in enumerate((70, 33, 129))]
+    Xd = dev_bf16(X)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+
+    def descs(shared):
+        out = []
+        for W in Ws:
+            N = W.shape[0]
+            out.append(dict(W=dev_bf16(W), X=Xd if shared else Xd.clone(),
+                            T01=torch.zeros(2, 16, dtype=torch.float32, device=DEV),
+                            scales=torch.empty(N, K // 16, dtype=torch.uint8, device=DEV),
+                            tensor_scale=torch.ones(1, dtype=torch.float32, device=DEV),
+                            ws=binding.alloc_workspace(NVFP4, N, K, X.shape[0]),
+                            T01_bf16=torch.empty(2, 16, dtype=torch.uint16, device=DEV),
+                            codes=torch.empty(N, K // 2, dtype=torch.uint8, device=DEV),
+                            err_out=torch.zeros(2, dtype=torch.float64, device=DEV)))
+        return out
+
+    counts = {}
+    for shared in (False, True):
+        d = descs(shared)
+        n0 = binding.launch_count()
+        binding.quantize_layers(d, NVFP4, n_outer=4, init=binding.INIT_QUANTILE, dev_status=status)
+        torch.cuda.synchronize()
+        counts[shared] = binding.launch_count() - n0
+        assert int(status.item()) == 0
+        for i, (W, r) in enumerate(zip(Ws, d)):
+            o = oracle.fit_layer(W, NVFP4, 16, 4, X=X, init="quantile")
+            assert table_close(host(r["T01"]), o["T"])[0]
+            check_end_to_end_bits(r, o, f"shared input {shared} layer {i}")
+            assert np.isclose(host(r["err_out"])[0], o["E_final"], rtol=1e-4)
+    assert counts[False] - counts[True] == 2 * (len(Ws) - 1), counts
+
+
 def test_quantize_layers_rejects_a_bad_output_before_enqueuing_anything():
     W, X = layer(NVFP4, 16, 256, name="qbatchbad")
     good = dict(W=dev_bf16(W), I=torch.ones(256, device=DEV), T01=torch.zeros(2, 16, device=DEV),
